@@ -1,0 +1,163 @@
+/*
+ * grass.h -- C ABI of the GRASS per-layer structured-sparse gradient step for
+ * NVIDIA B200 (sm_100a).
+ *
+ * GRASS (arXiv 2406.17660) trains a linear layer W (m x n) through a sparse
+ * projection P = (rho B)^T that keeps r of the m gradient rows.  With dY (T x m)
+ * the gradient w.r.t. the layer's outputs and X (T x n) its inputs, one
+ * iteration of the paper's Algorithm 1 is: every K iterations pick the rows
+ * (compute_P, Section 3.2); then G_C = P^T (dY^T X) without forming the m x n
+ * gradient (Section 3.1), Adam on the r x n state (Appendix A), and
+ * W <- W + alpha P Delta on the r picked rows only (Section 3.1).
+ *
+ * Conventions shared by every call
+ *   - Every pointer is a DEVICE pointer unless it is marked "host".  The caller
+ *     owns all buffers; the library allocates no device memory and keeps no
+ *     state between calls except an encoded-descriptor cache on the host and one
+ *     small per-device status word (see grass_device_status).
+ *   - Matrices are row-major; a leading dimension `ld*` is the row pitch in
+ *     ELEMENTS and must be >= the row length.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Calls only enqueue work and return; nothing synchronises except
+ *     grass_device_status.
+ *   - The return value is a grass_status_t.  Argument errors are detected on
+ *     the host, nothing is launched and no output is touched.  Conditions only
+ *     the device can see (degenerate norms, a row index outside [0, m), a wait
+ *     that ran out) are recorded in the status word and the affected outputs
+ *     are left unwritten where that is possible; no kernel traps or aborts.
+ *   - Rows are 0-based.  sigma (the paper's sigma_j) is int32 `idx[r]`, the
+ *     diagonal of rho is fp32 `rho[r]`: the "2r numbers" storage of P
+ *     (Section 3.1, "Efficient Storage of P").
+ */
+#ifndef GRASS_B200_H_
+#define GRASS_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GRASS_OK = 0,
+  GRASS_ERR_INVALID_ARG = 1, /* NULL pointer, bad size, r > m, ld < row length, idx out of range */
+  GRASS_ERR_ALIGNMENT = 2,   /* a pointer or pitch misses the alignment a path needs */
+  GRASS_ERR_UNSUPPORTED = 3, /* dtype or method this build does not implement */
+  GRASS_ERR_DEGENERATE = 4,  /* norms negative / non-finite, or all zero for a sampling method */
+  GRASS_ERR_WORKSPACE = 5,   /* workspace NULL, misaligned or smaller than *_workspace_bytes */
+  GRASS_ERR_CUDA = 6,        /* a CUDA runtime or driver call failed (see stderr) */
+  GRASS_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out */
+} grass_status_t;
+
+typedef enum { GRASS_F32 = 0, GRASS_BF16 = 1 } grass_dtype_t;
+
+typedef enum {
+  GRASS_SEL_TOPR = 0,            /* Section 3.2 B */
+  GRASS_SEL_MULTINOMIAL_NORM = 1 /* Section 3.2 A, Theorem 1 (with replacement) */
+} grass_sel_t;
+
+/*
+ * Row norms lambda_k = ||G[k, :]||_2 of a formed gradient (Section 3.2; the
+ * "mn" term of compute_P in the paper's summary table).
+ *   G      m x n, dtype `dt`, row pitch ldg; read only.
+ *   norms  [m] fp32, written.
+ * Accumulates in fp32.  Any alignment is accepted (128-bit loads are used when
+ * G and ldg allow them).
+ */
+int grass_row_norms(const void* G, int dt, int64_t m, int64_t n, int64_t ldg,
+                    float* norms, void* stream);
+
+/*
+ * compute_P (Section 3.2): choose sigma and rho from the row norms.
+ *   GRASS_SEL_TOPR: rho = 1, sigma = the r largest norms; equal norms go to
+ *     the lower row index.
+ *   GRASS_SEL_MULTINOMIAL_NORM: sigma_j i.i.d. ~ Multinomial(1, q), q_k =
+ *     lambda_k / sum(lambda), rho_j = 1 / sqrt(r q_{sigma_j}).  Draw j inverts
+ *     the fp64 running sum of the norms at u_j * sum, u_j = w_j * 2^-32, where
+ *     w_j is word (j mod 4) of Philox4x32-10 with key (seed low, seed high) and
+ *     counter (j div 4, layer_id, epoch, 0x47524153): sigma_j = min{k : c_k >
+ *     u_j * sum}.  The result is a pure function of (norms, seed, layer_id,
+ *     epoch); no generator state is kept.
+ *   norms  [m] fp32, read only.     idx [r] int32 and rho [r] fp32, written,
+ *   ascending by row (repeated rows are adjacent).
+ *   ws     scratch of at least grass_select_workspace_bytes(m, r, method)
+ *          bytes, 256-byte aligned; contents need not survive the call.
+ * 1 <= r <= m < 2^31.  If a norm is negative, NaN or infinite, or all are zero
+ * under a sampling method, idx and rho are left unwritten and the status word
+ * is set to GRASS_ERR_DEGENERATE.
+ */
+size_t grass_select_workspace_bytes(int64_t m, int32_t r, int method);
+int grass_select(const float* norms, int64_t m, int32_t r, int method, uint64_t seed,
+                 uint32_t layer_id, uint32_t epoch, int32_t* idx, float* rho, void* ws,
+                 size_t ws_bytes, void* stream);
+
+/*
+ * Projected gradient (Section 3.1, "Efficient Gradient Projection"):
+ *   Gc[j, c] = rho_j * sum_t dY[t, idx_j] * X[t, c],   j < r, c < n,
+ * i.e. rho ((B dY^T) X); the m x n gradient is never formed.
+ *   dY   T x m, pitch lddy;  X  T x n, pitch ldx;  both dtype `dt`, read only.
+ *   idx  [r] int32 rows in [0, m); may repeat.  NULL means the identity
+ *        (requires r == m): the call then returns the dense gradient dY^T X,
+ *        which is what a refresh iteration feeds to grass_row_norms.
+ *   rho  [r] fp32 or NULL (all ones).
+ *   Gc   r x n fp32, pitch ldgc, written.
+ *   ws   scratch of at least grass_project_workspace_bytes(T, m, n, r, dt)
+ *        bytes, 256-byte aligned.
+ * GRASS_BF16 runs on the tensor cores (bf16 products, fp32 accumulation) and
+ * needs X 16-byte aligned with ldx a multiple of 8 (and the same of dY / lddy
+ * when idx is NULL), else GRASS_ERR_ALIGNMENT.  GRASS_F32 uses fp32 FMA and
+ * accepts any alignment.  The sum over tokens is split into a fixed number of
+ * slices added in a fixed order: results are bit-reproducible run to run.
+ * A row index outside [0, m) contributes zeros and sets the status word.
+ */
+size_t grass_project_workspace_bytes(int64_t T, int64_t m, int64_t n, int32_t r, int dt);
+int grass_project_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx, int dt,
+                       int64_t T, int64_t m, int64_t n, const int32_t* idx, const float* rho,
+                       int32_t r, float* Gc, int64_t ldgc, void* ws, size_t ws_bytes,
+                       void* stream);
+
+/*
+ * adam.update on the subspace state (Appendix A):
+ *   M <- beta1 M + (1 - beta1) Gc;  V <- beta2 V + (1 - beta2) Gc^2;
+ *   U = -lr * (M / (1 - beta1^step)) / (sqrt(V / (1 - beta2^step)) + eps).
+ *   Gc r x n fp32 (pitch ldgc), read only.  M, V updated in place and U
+ *   written, all r x n fp32 with pitch ldstate.  U may alias Gc.
+ *   step >= 1 counts the updates since M and V were last zeroed (the paper's
+ *   update_state reset is a memset by the caller plus step = 1).
+ * Hyper-parameters are doubles so that 1 - beta is formed without first
+ * rounding beta to fp32; the element arithmetic is fp32.
+ */
+int grass_subspace_adam(const float* Gc, int64_t ldgc, float* M, float* V, float* U,
+                        int64_t ldstate, int32_t r, int64_t n, double lr, double beta1,
+                        double beta2, double eps, int32_t step, void* stream);
+
+/*
+ * Row-sparse apply (Algorithm 1 "Apply update"; Section 3.1 "Efficient Weight
+ * Update"):  W <- W + alpha P U, i.e. W[idx_j, :] += alpha * rho_j * U[j, :].
+ *   W    m x n, dtype wdt, pitch ldw, updated in place; rows not in idx are
+ *        not read or written.
+ *   U    r x n fp32, pitch ldu.   rho NULL = ones.
+ *   idx  [r] ascending (as grass_select writes it); repeated rows must be
+ *        adjacent: their terms are summed in fp32 in order of j and the row is
+ *        written once (bf16: one round-to-nearest-even at the end).
+ * A row index outside [0, m) is skipped and sets the status word.
+ */
+int grass_scatter_update(void* W, int wdt, int64_t m, int64_t n, int64_t ldw, const float* U,
+                         int64_t ldu, const int32_t* idx, const float* rho, int32_t r,
+                         double alpha, void* stream);
+
+/*
+ * Read and clear the current device's status word.  Synchronises `stream`.
+ * Returns GRASS_OK or the first error a kernel recorded since the last call;
+ * if detail (host pointer, may be NULL) is given it receives a kernel-specific
+ * value (the offending row index, or the stage a wait gave up in).
+ */
+int grass_device_status(void* stream, int32_t* detail);
+
+const char* grass_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRASS_B200_H_ */

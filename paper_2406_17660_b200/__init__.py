@@ -1,0 +1,15 @@
+"""GRASS structured-sparse gradient step for B200: Python binding over the C-ABI library.
+
+The CUDA library (libgrass_b200.so, built by `python -m paper_2406_17660_b200.build`)
+does all the work; this package only marshals torch tensors into pointers.
+Importing the package does not load the library; the first call does, and
+raises if it has not been built.
+"""
+from .binding import (  # noqa: F401
+    GrassError, BF16, F32, SEL_TOPR, SEL_MULTINOMIAL_NORM,
+    grass_row_norms, grass_select, grass_select_workspace_bytes,
+    grass_project_grad, grass_project_workspace_bytes,
+    grass_subspace_adam, grass_scatter_update, grass_device_status,
+    grass_status_string, library_path, load_library,
+)
+from .step import GrassLayer  # noqa: F401

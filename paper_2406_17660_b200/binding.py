@@ -1,0 +1,177 @@
+"""ctypes binding of include/grass.h: same names, torch tensors in place of pointers.
+
+Argument marshalling only.  Every function enqueues on torch's current CUDA
+stream and raises GrassError on a non-zero status; nothing here computes.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_double, c_int, c_int32, c_int64, c_size_t, c_uint32, c_uint64, c_void_p
+
+import torch
+
+F32, BF16 = 0, 1
+SEL_TOPR, SEL_MULTINOMIAL_NORM = 0, 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB = None
+
+
+class GrassError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {grass_status_string(status)} (status {status})")
+
+
+def library_path() -> str:
+    return os.path.join(_HERE, "libgrass_b200.so")
+
+
+_SIGNATURES = {
+    "grass_row_norms": (c_int, [c_void_p, c_int, c_int64, c_int64, c_int64, c_void_p, c_void_p]),
+    "grass_select_workspace_bytes": (c_size_t, [c_int64, c_int32, c_int]),
+    "grass_select": (c_int, [c_void_p, c_int64, c_int32, c_int, c_uint64, c_uint32, c_uint32,
+                             c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "grass_project_workspace_bytes": (c_size_t, [c_int64, c_int64, c_int64, c_int32, c_int]),
+    "grass_project_grad": (c_int, [c_void_p, c_int64, c_void_p, c_int64, c_int, c_int64, c_int64,
+                                   c_int64, c_void_p, c_void_p, c_int32, c_void_p, c_int64,
+                                   c_void_p, c_size_t, c_void_p]),
+    "grass_subspace_adam": (c_int, [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int64,
+                                    c_int32, c_int64, c_double, c_double, c_double, c_double,
+                                    c_int32, c_void_p]),
+    "grass_scatter_update": (c_int, [c_void_p, c_int, c_int64, c_int64, c_int64, c_void_p, c_int64,
+                                     c_void_p, c_void_p, c_int32, c_double, c_void_p]),
+    "grass_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int32)]),
+    "grass_status_string": (ctypes.c_char_p, [c_int]),
+}
+
+
+def load_library():
+    """Load libgrass_b200.so (once).  There is no fallback: a missing library is an error."""
+    global _LIB
+    if _LIB is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise RuntimeError(
+                f"{path} is missing: build it with `python -m paper_2406_17660_b200.build` "
+                "(needs nvcc); this package has no other execution path")
+        lib = ctypes.CDLL(path)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _LIB = lib
+    return _LIB
+
+
+def exported_symbols():
+    return sorted(_SIGNATURES)
+
+
+def grass_status_string(status: int) -> str:
+    return load_library().grass_status_string(int(status)).decode()
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _ld(t: torch.Tensor) -> int:
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError("expected a 2-D tensor with unit inner stride")
+    return t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+def _stream():
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise GrassError(status, where)
+
+
+def _require(t, dtype, name):
+    if t.dtype != dtype or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor of {dtype}")
+
+
+def grass_row_norms(G: torch.Tensor, norms: torch.Tensor) -> None:
+    m, n = G.shape
+    _require(norms, torch.float32, "norms")
+    _check(load_library().grass_row_norms(_ptr(G), _dtype_code(G), m, n, _ld(G), _ptr(norms),
+                                          _stream()), "grass_row_norms")
+
+
+def grass_select_workspace_bytes(m: int, r: int, method: int) -> int:
+    return int(load_library().grass_select_workspace_bytes(m, r, method))
+
+
+def grass_select(norms, r, method, seed, layer_id, epoch, idx, rho, ws) -> None:
+    _require(norms, torch.float32, "norms")
+    _require(idx, torch.int32, "idx")
+    _require(rho, torch.float32, "rho")
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(load_library().grass_select(_ptr(norms), norms.numel(), r, method, seed, layer_id, epoch,
+                                       _ptr(idx), _ptr(rho), _ptr(ws), ws_bytes, _stream()),
+           "grass_select")
+
+
+def grass_project_workspace_bytes(T: int, m: int, n: int, r: int, dt: int) -> int:
+    return int(load_library().grass_project_workspace_bytes(T, m, n, r, dt))
+
+
+def grass_project_grad(dY, X, idx, rho, r, Gc, ws) -> None:
+    T, m = dY.shape
+    T2, n = X.shape
+    if T2 != T or dY.dtype != X.dtype:
+        raise ValueError("dY and X must share the token dimension and dtype")
+    _require(Gc, torch.float32, "Gc")
+    if idx is not None:
+        _require(idx, torch.int32, "idx")
+    if rho is not None:
+        _require(rho, torch.float32, "rho")
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(load_library().grass_project_grad(_ptr(dY), _ld(dY), _ptr(X), _ld(X), _dtype_code(X), T,
+                                             m, n, _ptr(idx), _ptr(rho), r, _ptr(Gc), _ld(Gc),
+                                             _ptr(ws), ws_bytes, _stream()), "grass_project_grad")
+
+
+def grass_subspace_adam(Gc, M, V, U, lr, beta1, beta2, eps, step) -> None:
+    r, n = M.shape
+    for t, name in ((Gc, "Gc"), (M, "M"), (V, "V"), (U, "U")):
+        _require(t, torch.float32, name)
+    if _ld(V) != _ld(M) or _ld(U) != _ld(M):
+        raise ValueError("M, V and U must share one row pitch")
+    _check(load_library().grass_subspace_adam(_ptr(Gc), _ld(Gc), _ptr(M), _ptr(V), _ptr(U), _ld(M),
+                                              r, n, lr, beta1, beta2, eps, step, _stream()),
+           "grass_subspace_adam")
+
+
+def grass_scatter_update(W, U, idx, rho, alpha) -> None:
+    m, n = W.shape
+    r = idx.numel()
+    _require(U, torch.float32, "U")
+    _require(idx, torch.int32, "idx")
+    if rho is not None:
+        _require(rho, torch.float32, "rho")
+    _check(load_library().grass_scatter_update(_ptr(W), _dtype_code(W), m, n, _ld(W), _ptr(U),
+                                               _ld(U), _ptr(idx), _ptr(rho), r, alpha, _stream()),
+           "grass_scatter_update")
+
+
+def grass_device_status(raise_on_error: bool = True):
+    """Synchronise the current stream and return (status, detail) of the device status word."""
+    detail = c_int32(0)
+    status = load_library().grass_device_status(_stream(), ctypes.byref(detail))
+    if status != 0 and raise_on_error:
+        raise GrassError(status, f"device status (detail {detail.value})")
+    return status, detail.value

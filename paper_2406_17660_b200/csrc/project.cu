@@ -1,0 +1,226 @@
+// grass_project_grad: host side (argument checks, tiling plan, TMA descriptors,
+// launches).  The kernels are in project_tc.cuh (bf16, tcgen05) and
+// project_simt.cuh (fp32).
+#include <cudaTypedefs.h>
+
+#include "common.cuh"
+#include "project_simt.cuh"
+#include "project_tc.cuh"
+
+namespace grass {
+namespace {
+
+constexpr int kSmCount = 148;
+constexpr size_t kSmemBudget = 227 * 1024 - 1024;  // dynamic part; the rest holds the barriers
+
+struct TcPlan {
+  int r_pad;      // r_blocks * r_cta: width of the gathered operand
+  int r_cta, r_blocks;
+  int MB, n_blocks;
+  int k_blocks, split_k, stages;
+  size_t smem_bytes;
+  long long ld_part;        // pitch of a split-K partial, elements
+  size_t ag_bytes, part_bytes;
+};
+
+// Choose the CTA tile and the token split.  Cost model in SM clocks: the MMA
+// phase takes waves * (token blocks per CTA * clocks per block + prologue and
+// epilogue), and split-K partials cost their HBM write plus re-read.  Smaller
+// n-tiles (MB) make more, smaller CTAs, which cuts partial traffic when the
+// output is tiny; larger ones cut the number of times the gathered operand is
+// re-read.  The result depends only on (T, n, r), so it is reproducible.
+TcPlan make_plan(int64_t T, int64_t n, int r) {
+  TcPlan p;
+  const int r64 = static_cast<int>(round_up(static_cast<size_t>(r), 64));
+  p.r_blocks = (r64 + 511) / 512;
+  p.r_cta = static_cast<int>(round_up(static_cast<size_t>((r64 + p.r_blocks - 1) / p.r_blocks), 64));
+  p.r_pad = p.r_cta * p.r_blocks;
+  p.k_blocks = static_cast<int>((T + kTcBK - 1) / kTcBK);
+  int mb_max = 512 / p.r_cta;
+  mb_max = mb_max >= 4 ? 4 : (mb_max >= 2 ? 2 : 1);
+  while (mb_max > 1 && static_cast<int64_t>(mb_max / 2) * 128 >= n) mb_max /= 2;  // not past n
+
+  const double hbm_bytes_per_clk = 6.5e12 / 1.7e9;  // whole chip, per SM clock
+  double best = 1e300;
+  p.MB = 1;
+  p.split_k = 1;
+  for (int mb = mb_max; mb >= 1; mb /= 2) {
+    const int n_blocks = static_cast<int>((n + mb * 128 - 1) / (mb * 128));
+    const int64_t tiles = static_cast<int64_t>(n_blocks) * p.r_blocks;
+    const double clk_per_block = static_cast<double>(mb) * p.r_cta < 256.0
+                                     ? 256.0 : static_cast<double>(mb) * p.r_cta;
+    const double fixed = 2000.0 + mb * 128.0 * p.r_cta * 4.0 / 64.0;
+    const int max_s = p.k_blocks < 256 ? p.k_blocks : 256;
+    for (int s = 1; s <= max_s; ++s) {
+      const int64_t ctas = tiles * s;
+      const int64_t waves = (ctas + kSmCount - 1) / kSmCount;
+      const double blocks_per_cta = static_cast<double>((p.k_blocks + s - 1) / s);
+      double cost = waves * (blocks_per_cta * clk_per_block + fixed);
+      if (s > 1) cost += 8.0 * s * static_cast<double>(r) * n / hbm_bytes_per_clk;
+      if (cost < best) {
+        best = cost;
+        p.MB = mb;
+        p.split_k = s;
+      }
+    }
+  }
+  p.n_blocks = static_cast<int>((n + p.MB * 128 - 1) / (p.MB * 128));
+  const size_t stage_bytes = static_cast<size_t>(2 * p.MB + p.r_cta / 64) * kTcSlabBytes;
+  const int stages = static_cast<int>((kSmemBudget - 1024) / stage_bytes);
+  p.stages = stages > kTcMaxStages ? kTcMaxStages : stages;
+  p.smem_bytes = p.stages * stage_bytes + 1024;
+  p.ld_part = static_cast<long long>(round_up(static_cast<size_t>(n), 4));
+  p.ag_bytes = round_up(static_cast<size_t>(T) * p.r_pad * sizeof(__nv_bfloat16), 256);
+  p.part_bytes = p.split_k > 1
+                     ? round_up(static_cast<size_t>(p.split_k) * r * p.ld_part * sizeof(float), 256)
+                     : 0;
+  return p;
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows][cols] with row pitch ld (elements): box = {64 cols, 32 rows}, 128B swizzle.
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+  cuuint32_t box[2] = {64, static_cast<cuuint32_t>(kTcBK)};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult res = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
+                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (res != CUDA_SUCCESS) {
+    fprintf(stderr, "grass: cuTensorMapEncodeTiled failed with %d\n", static_cast<int>(res));
+    return false;
+  }
+  return true;
+}
+
+int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T, int64_t m,
+                 int64_t n, const int32_t* idx, const float* rho, int r, float* Gc, int64_t ldgc,
+                 void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (!aligned_to(X, 16) || ldx % 8 != 0) return GRASS_ERR_ALIGNMENT;
+  if (idx == nullptr && (!aligned_to(dY, 16) || lddy % 8 != 0)) return GRASS_ERR_ALIGNMENT;
+  const TcPlan plan = make_plan(T, n, r);
+  const bool gather = idx != nullptr;
+  const size_t need = (gather ? plan.ag_bytes : 0) + plan.part_bytes;
+  if (need > 0 && (ws == nullptr || !aligned_to(ws, 256) || ws_bytes < need))
+    return GRASS_ERR_WORKSPACE;
+  cudaError_t err;
+  int* status = status_word(&err);
+  if (status == nullptr) GRASS_CUDA_TRY(err);
+
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  GRASS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(kSmemBudget)));
+    attr_set[dev] = true;
+  }
+
+  char* wsp = static_cast<char*>(ws);
+  CUtensorMap tmX, tmA;
+  if (!make_map(&tmX, X, T, n, ldx)) return GRASS_ERR_CUDA;
+  if (gather) {
+    __nv_bfloat16* Ag = reinterpret_cast<__nv_bfloat16*>(wsp);
+    dim3 ggrid(static_cast<unsigned>((plan.r_pad / 8 + kGatherThreads - 1) / kGatherThreads),
+               static_cast<unsigned>((T + kGatherTokens - 1) / kGatherTokens));
+    gather_cols_kernel<<<ggrid, kGatherThreads, 0, s>>>(
+        static_cast<const __nv_bfloat16*>(dY), lddy, static_cast<int>(T), static_cast<int>(m), idx,
+        r, plan.r_pad, Ag, status);
+    GRASS_LAUNCH_CHECK();
+    if (!make_map(&tmA, Ag, T, plan.r_pad, plan.r_pad)) return GRASS_ERR_CUDA;
+    wsp += plan.ag_bytes;
+  } else {
+    if (!make_map(&tmA, dY, T, m, lddy)) return GRASS_ERR_CUDA;
+  }
+
+  TcParams p;
+  p.T = static_cast<int>(T);
+  p.n = static_cast<int>(n);
+  p.r = r;
+  p.r_cta = plan.r_cta;
+  p.MB = plan.MB;
+  p.stages = plan.stages;
+  p.k_blocks = plan.k_blocks;
+  p.split_k = plan.split_k;
+  p.status = status;
+  if (plan.split_k == 1) {
+    p.out = Gc;
+    p.ld_out = ldgc;
+    p.split_stride = 0;
+    p.rho = rho;
+  } else {
+    p.out = reinterpret_cast<float*>(wsp);
+    p.ld_out = plan.ld_part;
+    p.split_stride = static_cast<long long>(r) * plan.ld_part;
+    p.rho = nullptr;
+  }
+  dim3 grid(static_cast<unsigned>(plan.n_blocks), static_cast<unsigned>(plan.r_blocks),
+            static_cast<unsigned>(plan.split_k));
+  project_tc_kernel<<<grid, kTcThreads, plan.smem_bytes, s>>>(tmX, tmA, p);
+  GRASS_LAUNCH_CHECK();
+  if (plan.split_k > 1) {
+    const int vec = (n % 4 == 0) && (ldgc % 4 == 0) && aligned_to(Gc, 16);
+    const long long work = static_cast<long long>(r) * (vec ? n / 4 : n);
+    long long blocks = (work + 255) / 256;
+    if (blocks > kSmCount * 8) blocks = kSmCount * 8;
+    splitk_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(
+        p.out, plan.ld_part, p.split_stride, plan.split_k, r, static_cast<int>(n), rho, Gc, ldgc,
+        vec);
+    GRASS_LAUNCH_CHECK();
+  }
+  return GRASS_OK;
+}
+
+}  // namespace
+}  // namespace grass
+
+extern "C" size_t grass_project_workspace_bytes(int64_t T, int64_t m, int64_t n, int32_t r,
+                                                int dt) {
+  (void)m;
+  if (T < 1 || n < 1 || r < 1) return 0;
+  if (dt != GRASS_BF16) return 256;
+  const grass::TcPlan plan = grass::make_plan(T, n, r);
+  return plan.ag_bytes + plan.part_bytes + 256;
+}
+
+extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx, int dt,
+                                  int64_t T, int64_t m, int64_t n, const int32_t* idx,
+                                  const float* rho, int32_t r, float* Gc, int64_t ldgc, void* ws,
+                                  size_t ws_bytes, void* stream) {
+  using namespace grass;
+  if (dY == nullptr || X == nullptr || Gc == nullptr || T < 1 || m < 1 || n < 1 || r < 1 ||
+      lddy < m || ldx < n || ldgc < n || T > 0x7fffffffLL || m > 0x7fffffffLL ||
+      n > 0x7fffffffLL)
+    return GRASS_ERR_INVALID_ARG;
+  if (idx == nullptr && r != m) return GRASS_ERR_INVALID_ARG;
+  if (r > m) return GRASS_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dt == GRASS_BF16)
+    return project_bf16(dY, lddy, X, ldx, T, m, n, idx, rho, r, Gc, ldgc, ws, ws_bytes, s);
+  if (dt != GRASS_F32) return GRASS_ERR_UNSUPPORTED;
+  cudaError_t err;
+  int* status = status_word(&err);
+  if (status == nullptr) GRASS_CUDA_TRY(err);
+  dim3 grid(static_cast<unsigned>((n + kSimtBC - 1) / kSimtBC),
+            static_cast<unsigned>((r + kSimtBJ - 1) / kSimtBJ));
+  project_simt_kernel<float><<<grid, kSimtThreads, 0, s>>>(
+      static_cast<const float*>(dY), lddy, static_cast<const float*>(X), ldx, T, m, n, idx, rho, r,
+      Gc, ldgc, status);
+  GRASS_LAUNCH_CHECK();
+  return GRASS_OK;
+}

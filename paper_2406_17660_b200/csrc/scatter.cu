@@ -1,0 +1,126 @@
+// grass_scatter_update: W <- W + alpha P U on the r selected rows only
+// (Algorithm 1 "Apply update"; Section 3.1 "Efficient Weight Update").
+//
+// HBM-bound: per selected element 4 bytes of U in, one W element in and out.
+// idx is ascending, so repeated rows are adjacent.  The first j of each run of
+// equal rows owns the row: it sums alpha*rho_j*U[j,:] over its run in fp32, in
+// order of j, and writes the row once -- no atomics, bit-reproducible.
+#include "common.cuh"
+
+namespace grass {
+namespace {
+
+constexpr int kThreads = 256;
+
+template <typename T> struct WTraits;
+template <> struct WTraits<float> {
+  static constexpr int N = 4;
+  using vec = float4;
+  static __device__ __forceinline__ void add_store(float* w, const float* acc) {
+    float4 v = *reinterpret_cast<float4*>(w);
+    v.x += acc[0]; v.y += acc[1]; v.z += acc[2]; v.w += acc[3];
+    *reinterpret_cast<float4*>(w) = v;
+  }
+  static __device__ __forceinline__ float add1(float w, float a) { return w + a; }
+};
+template <> struct WTraits<__nv_bfloat16> {
+  static constexpr int N = 8;
+  using vec = uint4;
+  static __device__ __forceinline__ void add_store(__nv_bfloat16* w, const float* acc) {
+    uint4 raw = *reinterpret_cast<uint4*>(w);
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 f = __bfloat1622float2(h[i]);
+      f.x += acc[2 * i];
+      f.y += acc[2 * i + 1];
+      h[i] = __floats2bfloat162_rn(f.x, f.y);
+    }
+    *reinterpret_cast<uint4*>(w) = raw;
+  }
+  static __device__ __forceinline__ __nv_bfloat16 add1(__nv_bfloat16 w, float a) {
+    return __float2bfloat16_rn(__bfloat162float(w) + a);
+  }
+};
+
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(kThreads)
+scatter_kernel(T* __restrict__ W, int64_t m, int64_t n, int64_t ldw, const float* __restrict__ U,
+               int64_t ldu, const int32_t* __restrict__ idx, const float* __restrict__ rho, int r,
+               float alpha, int* status) {
+  const int j0 = blockIdx.y;
+  const int row = idx[j0];
+  if (j0 > 0 && idx[j0 - 1] == row) return;  // not the head of its run
+  if (row < 0 || row >= m) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) record_status(status, GRASS_ERR_INVALID_ARG, row);
+    return;
+  }
+  constexpr int N = WTraits<T>::N;
+  T* w = W + static_cast<int64_t>(row) * ldw;
+  if (VEC) {
+    const int64_t c = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) * N;
+    if (c >= n) return;
+    float acc[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) acc[i] = 0.f;
+    for (int j = j0; j < r && idx[j] == row; ++j) {
+      const float s = alpha * (rho != nullptr ? rho[j] : 1.f);
+      const float4* u = reinterpret_cast<const float4*>(U + static_cast<int64_t>(j) * ldu + c);
+#pragma unroll
+      for (int q = 0; q < N / 4; ++q) {
+        const float4 v = __ldg(u + q);
+        acc[4 * q + 0] += s * v.x;
+        acc[4 * q + 1] += s * v.y;
+        acc[4 * q + 2] += s * v.z;
+        acc[4 * q + 3] += s * v.w;
+      }
+    }
+    WTraits<T>::add_store(w + c, acc);
+  } else {
+    const int64_t c0 = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) * N;
+    for (int64_t c = c0; c < c0 + N && c < n; ++c) {
+      float acc = 0.f;
+      for (int j = j0; j < r && idx[j] == row; ++j)
+        acc += alpha * (rho != nullptr ? rho[j] : 1.f) * U[static_cast<int64_t>(j) * ldu + c];
+      w[c] = WTraits<T>::add1(w[c], acc);
+    }
+  }
+}
+
+template <typename T>
+int launch(void* W, int64_t m, int64_t n, int64_t ldw, const float* U, int64_t ldu,
+           const int32_t* idx, const float* rho, int r, float alpha, cudaStream_t s) {
+  constexpr int N = WTraits<T>::N;
+  cudaError_t err;
+  int* status = status_word(&err);
+  if (status == nullptr) GRASS_CUDA_TRY(err);
+  const bool vec = (n % N == 0) && (ldw % N == 0) && (ldu % 4 == 0) && aligned_to(W, 16) &&
+                   aligned_to(U, 16);
+  dim3 grid(static_cast<unsigned>((n + kThreads * N - 1) / (kThreads * N)),
+            static_cast<unsigned>(r));
+  if (vec)
+    scatter_kernel<T, true><<<grid, kThreads, 0, s>>>(static_cast<T*>(W), m, n, ldw, U, ldu, idx,
+                                                      rho, r, alpha, status);
+  else
+    scatter_kernel<T, false><<<grid, kThreads, 0, s>>>(static_cast<T*>(W), m, n, ldw, U, ldu, idx,
+                                                       rho, r, alpha, status);
+  GRASS_LAUNCH_CHECK();
+  return GRASS_OK;
+}
+
+}  // namespace
+}  // namespace grass
+
+extern "C" int grass_scatter_update(void* W, int wdt, int64_t m, int64_t n, int64_t ldw,
+                                    const float* U, int64_t ldu, const int32_t* idx,
+                                    const float* rho, int32_t r, double alpha, void* stream) {
+  if (W == nullptr || U == nullptr || idx == nullptr || m < 1 || n < 1 || r < 1 || ldw < n ||
+      ldu < n || r > 65535 || m > 0x7fffffffLL)
+    return GRASS_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const float a = static_cast<float>(alpha);
+  if (wdt == GRASS_F32) return grass::launch<float>(W, m, n, ldw, U, ldu, idx, rho, r, a, s);
+  if (wdt == GRASS_BF16)
+    return grass::launch<__nv_bfloat16>(W, m, n, ldw, U, ldu, idx, rho, r, a, s);
+  return GRASS_ERR_UNSUPPORTED;
+}

@@ -1,0 +1,264 @@
+// grass_select: compute_P of the GRASS paper (Section 3.2) -- Top-r, or
+// Multinomial-Norm sampling with replacement and rho_j = 1/sqrt(r q_sigma_j).
+//
+// m is at most a few tens of thousands and r at most a few thousand, so this
+// is a latency-bound single-CTA kernel (1024 threads); everything it needs to
+// agree on is agreed on through shared memory and block-wide scans, and the
+// output order (ascending row) is produced by scans in row order, so the
+// result does not depend on thread scheduling.
+//
+//   Top-r: the fp32 bit pattern of a non-negative float orders like the float,
+//   so the r-th largest norm is found by a 4-pass, 8-bit-digit radix select.
+//   Rows above the threshold are taken; rows equal to it are taken lowest row
+//   first until r are chosen.
+//
+//   Multinomial-Norm: fp64 inclusive running sum of the norms (block scan in
+//   row order), then one thread per draw: Philox4x32-10 word -> u -> binary
+//   search for min{k : c_k > u S}; hits are counted per row with integer
+//   atomics (order-independent), and a last scan over the counts writes the
+//   rows in ascending order with their rho.
+#include "common.cuh"
+
+namespace grass {
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+constexpr uint32_t kStreamTag = 0x47524153u;
+
+// ---- Philox4x32-10 (Salmon et al., SC'11) ----
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+    k.x += 0x9E3779B9u;
+    k.y += 0xBB67AE85u;
+  }
+  return c;
+}
+
+// Inclusive block scan over kThreads values; returns this thread's inclusive
+// prefix and sets `total` for all threads.  `scratch` holds kWarps + 1 values.
+template <typename T>
+__device__ __forceinline__ T block_inclusive_scan(T v, T* scratch, T& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    T up = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v += up;
+  }
+  __syncthreads();  // scratch may still be read from a previous call
+  if (lane == 31) scratch[warp] = v;
+  __syncthreads();
+  if (warp == 0) {
+    T w = lane < kWarps ? scratch[lane] : T(0);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      T up = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += up;
+    }
+    if (lane < kWarps) scratch[lane] = w;
+  }
+  __syncthreads();
+  total = scratch[kWarps - 1];
+  return warp == 0 ? v : v + scratch[warp - 1];
+}
+
+__device__ __forceinline__ uint32_t norm_key(float v) {
+  return v == 0.f ? 0u : __float_as_uint(v);  // folds -0 into +0
+}
+
+struct SelectArgs {
+  const float* norms;
+  int m, r, method;
+  uint32_t seed_lo, seed_hi, layer_id, epoch;
+  int32_t* idx;
+  float* rho;
+  double* cdf;    // [m]   (sampling methods)
+  int* counts;    // [m]   (sampling methods)
+  int* status;
+};
+
+__global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
+  __shared__ int s_hist[256];
+  __shared__ int s_int[kWarps + 1];
+  __shared__ double s_dbl[kWarps + 1];
+  __shared__ int s_flag;
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_need;
+  const int tid = threadIdx.x;
+  const int m = a.m, r = a.r;
+
+  // ---- validate: every norm finite and >= 0 ----
+  if (tid == 0) s_flag = 0;
+  __syncthreads();
+  {
+    int bad = 0;
+    for (int k = tid; k < m; k += kThreads) {
+      const float v = a.norms[k];
+      if (!(v >= 0.f) || isinf(v)) bad = k + 1;
+    }
+    if (bad) atomicMax(&s_flag, bad);
+  }
+  __syncthreads();
+  if (s_flag != 0) {
+    if (tid == 0) record_status(a.status, GRASS_ERR_DEGENERATE, s_flag - 1);
+    return;
+  }
+
+  if (a.method == GRASS_SEL_TOPR) {
+    // ---- radix select of the r-th largest key ----
+    if (tid == 0) { s_prefix = 0u; s_need = r; }
+    for (int pass = 3; pass >= 0; --pass) {
+      const int shift = pass * 8;
+      if (tid < 256) s_hist[tid] = 0;
+      __syncthreads();
+      const uint32_t prefix = s_prefix;
+      const uint32_t himask = pass == 3 ? 0u : (0xffffffffu << (shift + 8));
+      for (int k = tid; k < m; k += kThreads) {
+        const uint32_t key = norm_key(a.norms[k]);
+        if ((key & himask) == prefix) atomicAdd(&s_hist[(key >> shift) & 0xff], 1);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int need = s_need, d = 255;
+        for (; d > 0; --d) {
+          if (s_hist[d] >= need) break;
+          need -= s_hist[d];
+        }
+        s_need = need;                       // how many to take among keys with this digit
+        s_prefix = prefix | (static_cast<uint32_t>(d) << shift);
+      }
+      __syncthreads();
+    }
+    const uint32_t tau = s_prefix;           // key of the r-th largest norm
+    const int need_eq = s_need;              // rows equal to tau to take, lowest row first
+    // ---- emit in ascending row order ----
+    int eq_base = 0, out_base = 0;
+    for (int k0 = 0; k0 < m; k0 += kThreads) {
+      const int k = k0 + tid;
+      uint32_t key = 0u;
+      int is_eq = 0, is_gt = 0;
+      if (k < m) {
+        key = norm_key(a.norms[k]);
+        is_eq = key == tau;
+        is_gt = key > tau;
+      }
+      int eq_total, sel_total;
+      const int eq_incl = block_inclusive_scan<int>(is_eq, s_int, eq_total);
+      const int sel = is_gt || (is_eq && (eq_base + eq_incl - 1) < need_eq);
+      const int sel_incl = block_inclusive_scan<int>(sel, s_int, sel_total);
+      if (sel) {
+        const int pos = out_base + sel_incl - 1;
+        a.idx[pos] = k;
+        a.rho[pos] = 1.f;
+      }
+      eq_base += eq_total;
+      out_base += sel_total;
+    }
+    return;
+  }
+
+  // ---- Multinomial-Norm ----
+  double carry = 0.0;
+  for (int k0 = 0; k0 < m; k0 += kThreads) {
+    const int k = k0 + tid;
+    const double v = k < m ? static_cast<double>(a.norms[k]) : 0.0;
+    double total;
+    const double incl = block_inclusive_scan<double>(v, s_dbl, total);
+    if (k < m) {
+      a.cdf[k] = carry + incl;
+      a.counts[k] = 0;
+    }
+    carry += total;
+  }
+  const double S = carry;
+  if (!(S > 0.0)) {
+    if (tid == 0) record_status(a.status, GRASS_ERR_DEGENERATE, -1);
+    return;
+  }
+  __syncthreads();  // cdf and counts visible block-wide (same CTA: global writes + barrier)
+  for (int j = tid; j < r; j += kThreads) {
+    const uint4 blk = philox4x32_10(make_uint4(static_cast<uint32_t>(j >> 2), a.layer_id, a.epoch,
+                                               kStreamTag),
+                                    make_uint2(a.seed_lo, a.seed_hi));
+    const uint32_t sel = j & 3;
+    const uint32_t word = sel == 0 ? blk.x : sel == 1 ? blk.y : sel == 2 ? blk.z : blk.w;
+    const double target = (static_cast<double>(word) * 0x1p-32) * S;
+    int lo = 0, hi = m - 1;                  // first k with cdf[k] > target
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (a.cdf[mid] > target) hi = mid; else lo = mid + 1;
+    }
+    atomicAdd(&a.counts[lo], 1);
+  }
+  __syncthreads();
+  int out_base = 0;
+  for (int k0 = 0; k0 < m; k0 += kThreads) {
+    const int k = k0 + tid;
+    const int cnt = k < m ? a.counts[k] : 0;
+    int total;
+    const int incl = block_inclusive_scan<int>(cnt, s_int, total);
+    if (cnt > 0) {
+      const double q = static_cast<double>(a.norms[k]) / S;
+      const float rho = static_cast<float>(1.0 / sqrt(static_cast<double>(r) * q));
+      const int pos = out_base + incl - cnt;
+      for (int i = 0; i < cnt; ++i) {
+        a.idx[pos + i] = k;
+        a.rho[pos + i] = rho;
+      }
+    }
+    out_base += total;
+  }
+}
+
+size_t cdf_bytes(int64_t m) { return round_up(static_cast<size_t>(m) * sizeof(double), 256); }
+
+}  // namespace
+}  // namespace grass
+
+extern "C" size_t grass_select_workspace_bytes(int64_t m, int32_t r, int method) {
+  (void)r;
+  if (m < 1) return 0;
+  if (method == GRASS_SEL_TOPR) return 256;  // unused, but never zero so callers can allocate
+  return grass::cdf_bytes(m) + grass::round_up(static_cast<size_t>(m) * sizeof(int), 256);
+}
+
+extern "C" int grass_select(const float* norms, int64_t m, int32_t r, int method, uint64_t seed,
+                            uint32_t layer_id, uint32_t epoch, int32_t* idx, float* rho, void* ws,
+                            size_t ws_bytes, void* stream) {
+  using namespace grass;
+  if (norms == nullptr || idx == nullptr || rho == nullptr || m < 1 || m > 0x7fffffffLL ||
+      r < 1 || r > m)
+    return GRASS_ERR_INVALID_ARG;
+  if (method != GRASS_SEL_TOPR && method != GRASS_SEL_MULTINOMIAL_NORM)
+    return GRASS_ERR_UNSUPPORTED;
+  SelectArgs a;
+  a.cdf = nullptr;
+  a.counts = nullptr;
+  if (method != GRASS_SEL_TOPR) {
+    if (ws == nullptr || !aligned_to(ws, 256) ||
+        ws_bytes < grass_select_workspace_bytes(m, r, method))
+      return GRASS_ERR_WORKSPACE;
+    a.cdf = static_cast<double*>(ws);
+    a.counts = reinterpret_cast<int*>(static_cast<char*>(ws) + cdf_bytes(m));
+  }
+  cudaError_t err;
+  a.status = status_word(&err);
+  if (a.status == nullptr) GRASS_CUDA_TRY(err);
+  a.norms = norms;
+  a.m = static_cast<int>(m);
+  a.r = r;
+  a.method = method;
+  a.seed_lo = static_cast<uint32_t>(seed & 0xffffffffu);
+  a.seed_hi = static_cast<uint32_t>(seed >> 32);
+  a.layer_id = layer_id;
+  a.epoch = epoch;
+  a.idx = idx;
+  a.rho = rho;
+  select_kernel<<<1, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  GRASS_LAUNCH_CHECK();
+  return GRASS_OK;
+}

@@ -1,0 +1,78 @@
+"""Host-only checks of the C ABI: the library builds, loads without a GPU, exports every
+symbol include/grass.h declares, and rejects bad arguments before touching the device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+from paper_2406_17660_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    entry.build()
+    return binding.load_library()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "grass.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(grass_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported_and_bound(lib):
+    names = _declared()
+    assert "grass_project_grad" in names and len(names) >= 9
+    for name in names:
+        assert hasattr(lib, name), name
+    assert set(names) == set(binding.exported_symbols())
+
+
+def test_status_strings(lib):
+    assert binding.grass_status_string(0) == "ok"
+    seen = {binding.grass_status_string(i) for i in range(8)}
+    assert len(seen) == 8 and "unknown status" not in seen
+    assert binding.grass_status_string(99) == "unknown status"
+
+
+def test_argument_errors_are_returned_without_a_device(lib):
+    null = ctypes.c_void_p(None)
+    fake = ctypes.c_void_p(0x1000)          # never dereferenced: checks fail first
+    assert lib.grass_row_norms(null, 0, 4, 4, 4, fake, null) == 1
+    assert lib.grass_row_norms(fake, 0, 4, 4, 3, fake, null) == 1            # ld < n
+    assert lib.grass_row_norms(fake, 7, 4, 4, 4, fake, null) == 3            # dtype
+    assert lib.grass_select(fake, 10, 11, 0, 0, 0, 0, fake, fake, null, 0, null) == 1   # r > m
+    assert lib.grass_select(fake, 10, 0, 0, 0, 0, 0, fake, fake, null, 0, null) == 1
+    assert lib.grass_select(fake, 10, 5, 9, 0, 0, 0, fake, fake, null, 0, null) == 3    # method
+    assert lib.grass_select(fake, 10, 5, 1, 0, 0, 0, fake, fake, null, 0, null) == 5    # no workspace
+    assert lib.grass_project_grad(fake, 8, fake, 8, 1, 16, 8, 8, null, null, 4, fake, 8, null, 0,
+                                  null) == 1                                 # idx NULL but r != m
+    assert lib.grass_project_grad(fake, 8, fake, 8, 1, 16, 8, 8, fake, null, 9, fake, 8, null, 0,
+                                  null) == 1                                 # r > m
+    assert lib.grass_project_grad(fake, 8, fake, 4, 1, 16, 8, 8, fake, null, 4, fake, 8, null, 0,
+                                  null) == 1                                 # ldx < n
+    assert lib.grass_project_grad(fake, 8, fake, 12, 1, 16, 8, 8, fake, null, 4, fake, 8, null, 0,
+                                  null) == 2                                 # bf16 pitch not 16-byte
+    assert lib.grass_project_grad(fake, 8, fake, 8, 1, 16, 8, 8, fake, null, 4, fake, 8, null, 0,
+                                  null) == 5                                 # bf16 needs workspace
+    assert lib.grass_subspace_adam(fake, 8, fake, fake, fake, 8, 4, 8, 1e-3, 0.9, 0.999, 1e-8, 0,
+                                   null) == 1                                # step < 1
+    assert lib.grass_subspace_adam(fake, 8, fake, fake, fake, 8, 4, 8, 1e-3, 1.0, 0.999, 1e-8, 1,
+                                   null) == 1                                # beta1 = 1
+    assert lib.grass_scatter_update(fake, 1, 8, 8, 8, fake, 8, null, null, 4, 0.25, null) == 1
+    assert lib.grass_scatter_update(fake, 5, 8, 8, 8, fake, 8, fake, null, 4, 0.25, null) == 3
+
+
+def test_workspace_queries_are_host_only_and_monotone(lib):
+    assert binding.grass_select_workspace_bytes(4096, 256, binding.SEL_TOPR) >= 256
+    a = binding.grass_select_workspace_bytes(4096, 256, binding.SEL_MULTINOMIAL_NORM)
+    assert a >= 4096 * 12
+    small = binding.grass_project_workspace_bytes(1024, 512, 512, 128, binding.BF16)
+    big = binding.grass_project_workspace_bytes(32768, 4096, 4096, 1024, binding.BF16)
+    assert 1024 * 128 * 2 <= small < big
+    assert big >= 32768 * 1024 * 2
+    assert binding.grass_project_workspace_bytes(1024, 512, 512, 128, binding.F32) == 256

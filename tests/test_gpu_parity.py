@@ -1,0 +1,326 @@
+"""Parity of the CUDA library (through the C ABI) with the fp64 oracle, element by element.
+
+Tolerances (stated by the build's acceptance criteria, and where tighter,
+derived from the arithmetic):
+  indices            bit-exact, except where the deciding fp64 quantity is within 1e-6 relative
+  projected gradient relative Frobenius error <= 1e-2 for bf16 inputs (acceptance); the kernel
+                     multiplies bf16 exactly and accumulates in fp32, so <= 1e-4 is also required
+                     (catches a dropped token block that 1e-2 would let through); fp32 path 1e-5
+  Adam M, V, U       1e-5 relative
+  updated rows       fp32 W: 1e-5 relative; bf16 W: at most 1 bf16 ulp from the oracle's rounding
+  unselected rows    bit-identical
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2406_17660_b200 as grass
+from paper_2406_17660_b200 import synthetic as syn
+from oracle import grass_oracle as oracle
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def rel_fro(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    return np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300)
+
+
+def f64(t):
+    return t.detach().to("cpu", torch.float32).numpy().astype(np.float64)
+
+
+def ws_bytes(nbytes):
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=DEV)
+
+
+# --------------------------------------------------------------------------- row norms
+@pytest.mark.parametrize("m,n,ld,dtype", [
+    (256, 256, 256, torch.float32),
+    (37, 1001, 1001, torch.float32),       # no 128-bit path, ragged
+    (64, 5461, 5464, torch.float32),       # padded pitch, tail columns
+    (24, 11008, 11008, torch.float32),     # CTA-per-row path
+    (9, 4099, 4104, torch.bfloat16),
+    (300, 520, 520, torch.bfloat16),
+    (1, 1, 1, torch.float32),
+])
+def test_row_norms(m, n, ld, dtype):
+    g = torch.Generator().manual_seed(m * 7 + n)
+    G = (torch.randn((m, n), generator=g) * torch.exp(torch.randn((m, 1), generator=g))).to(dtype)
+    Gd = syn._padded(G.to(DEV), ld)
+    norms = torch.full((m,), -1.0, dtype=torch.float32, device=DEV)
+    grass.grass_row_norms(Gd, norms)
+    grass.grass_device_status()
+    want = oracle.row_norms(f64(G))
+    np.testing.assert_allclose(f64(norms), want, rtol=1e-5, atol=0)
+
+
+# --------------------------------------------------------------------------- selection
+def _gpu_select(norms_np, r, method, seed=0, layer_id=0, epoch=0):
+    norms = torch.tensor(norms_np, dtype=torch.float32, device=DEV)
+    m = norms.numel()
+    idx = torch.full((r,), -7, dtype=torch.int32, device=DEV)
+    rho = torch.full((r,), -7.0, dtype=torch.float32, device=DEV)
+    ws = ws_bytes(grass.grass_select_workspace_bytes(m, r, method))
+    grass.grass_select(norms, r, method, seed, layer_id, epoch, idx, rho, ws)
+    status, detail = grass.grass_device_status(raise_on_error=False)
+    return status, idx.cpu().numpy(), rho.cpu().numpy()
+
+
+def _lognormal_norms(m, seed, zeros=0):
+    rng = np.random.default_rng(seed)
+    lam = np.exp(rng.standard_normal(m)).astype(np.float32)
+    if zeros:
+        lam[rng.choice(m, zeros, replace=False)] = 0.0
+    return lam
+
+
+@pytest.mark.parametrize("m,r", [(256, 32), (512, 128), (1000, 1), (1000, 1000), (13824, 1024),
+                                 (5000, 4097)])
+def test_select_topr_bit_exact(m, r):
+    lam = _lognormal_norms(m, m + r, zeros=m // 10)
+    status, idx, rho = _gpu_select(lam, r, grass.SEL_TOPR)
+    assert status == 0
+    sigma, _ = oracle.select_topr(lam, r)
+    assert np.array_equal(idx, sigma)
+    assert np.all(rho == 1.0)
+
+
+def test_select_topr_ties_lowest_index():
+    lam = np.zeros(3000, dtype=np.float32)
+    lam[5::7] = 2.0          # many equal norms straddling the threshold
+    lam[100] = 3.0
+    lam[2999] = 3.0
+    lam[0] = -0.0
+    for r in (1, 2, 3, 50, 400, 431, 2000):
+        status, idx, _ = _gpu_select(lam, r, grass.SEL_TOPR)
+        assert status == 0
+        assert np.array_equal(idx, oracle.select_topr(lam, r)[0]), r
+
+
+def _check_multinomial(lam, r, seed, layer_id, epoch):
+    status, idx, rho = _gpu_select(lam, r, grass.SEL_MULTINOMIAL_NORM, seed, layer_id, epoch)
+    assert status == 0
+    sigma, rho_ref = oracle.select_multinomial_norm(lam, r, seed, layer_id, epoch)
+    if not np.array_equal(idx, sigma):
+        # allowed only where a draw falls within 1e-6 (relative to the total) of a CDF step
+        c = np.cumsum(lam.astype(np.float64))
+        u = oracle.draw_words(r, seed, layer_id, epoch).astype(np.float64) * 2.0 ** -32 * c[-1]
+        gap = np.min(np.abs(c[None, :] - u[:, None]), axis=1) / c[-1]
+        assert np.sum(idx != sigma) <= np.sum(gap < 1e-6), "index mismatch beyond the near-tie allowance"
+    else:
+        np.testing.assert_allclose(rho, rho_ref, rtol=1e-6)
+    assert np.all(np.diff(idx) >= 0)
+
+
+@pytest.mark.parametrize("m,r,seed,layer_id,epoch", [
+    (512, 128, 0, 0, 0), (512, 128, 0, 3, 17), (1376, 128, 12345678901234567, 55, 2),
+    (13824, 1024, 7, 1, 1), (300, 300, 99, 0, 0), (2048, 512, 2 ** 63 + 5, 167, 4000000000),
+    (64, 1, 1, 1, 1),
+])
+def test_select_multinomial_matches_oracle(m, r, seed, layer_id, epoch):
+    _check_multinomial(_lognormal_norms(m, m * 3 + r, zeros=m // 8), r, seed, layer_id, epoch)
+
+
+def test_select_degenerate_inputs_leave_outputs_untouched():
+    lam = _lognormal_norms(100, 1)
+    for bad, method in ((np.nan, grass.SEL_TOPR), (np.inf, grass.SEL_TOPR), (-1.0, grass.SEL_TOPR),
+                        (np.nan, grass.SEL_MULTINOMIAL_NORM)):
+        x = lam.copy()
+        x[41] = bad
+        status, idx, rho = _gpu_select(x, 10, method)
+        assert status == 4                       # GRASS_ERR_DEGENERATE
+        assert np.all(idx == -7) and np.all(rho == -7.0)
+    status, idx, rho = _gpu_select(np.zeros(100, dtype=np.float32), 10, grass.SEL_MULTINOMIAL_NORM)
+    assert status == 4 and np.all(idx == -7)
+    status, idx, _ = _gpu_select(np.zeros(100, dtype=np.float32), 10, grass.SEL_TOPR)
+    assert status == 0 and np.array_equal(idx, np.arange(10))
+
+
+# --------------------------------------------------------------------------- projection
+def _project_case(T, m, n, r, dtype, seed, ldx=None, lddy=None, identity=False, dup=False,
+                  with_rho=True):
+    X = syn.make_X(T, n, dtype, seed0=seed, ld=ldx)
+    dY = syn.make_dY(T, m, dtype, seed0=seed, ld=lddy)
+    rng = np.random.default_rng(seed)
+    if identity:
+        sigma, idx_t = np.arange(m), None
+        r = m
+    else:
+        sigma = np.sort(rng.choice(m, r, replace=dup))
+        idx_t = torch.tensor(sigma, dtype=torch.int32, device=DEV)
+    rho_np = (0.5 + rng.random(r)).astype(np.float32) if with_rho else None
+    rho_t = None if rho_np is None else torch.tensor(rho_np, device=DEV)
+    Xd = syn._padded(X.to(DEV), ldx or n)
+    dYd = syn._padded(dY.to(DEV), lddy or m)
+    Gc = torch.full((r, n), float("nan"), dtype=torch.float32, device=DEV)
+    dt = grass.BF16 if dtype == torch.bfloat16 else grass.F32
+    ws = ws_bytes(grass.grass_project_workspace_bytes(T, m, n, r, dt))
+    grass.grass_project_grad(dYd, Xd, idx_t, rho_t, r, Gc, ws)
+    grass.grass_device_status()
+    want = oracle.project_grad(f64(dY), f64(X), sigma, rho_np)
+    return f64(Gc), want
+
+
+@pytest.mark.parametrize("T,m,n,r", [(512, 256, 256, 32), (100, 50, 70, 7), (33, 65, 129, 65)])
+def test_project_fp32(T, m, n, r):
+    got, want = _project_case(T, m, n, r, torch.float32, seed=T + r, dup=(r == 7))
+    assert rel_fro(got, want) <= 1e-5
+    got, want = _project_case(T, m, n, r, torch.float32, seed=T, identity=True, with_rho=False)
+    assert rel_fro(got, want) <= 1e-5
+
+
+@pytest.mark.parametrize("T,m,n,r,ldx,kw", [
+    (256, 256, 256, 64, None, {}),                       # one tile, 8 token blocks
+    (1000, 300, 328, 100, None, {}),                     # ragged T, n, r
+    (4096, 512, 512, 128, None, {"dup": True}),          # 60M-shaped, repeated rows
+    (2048, 1376, 512, 128, None, {}),
+    (3000, 1024, 2736, 256, None, {}),                   # 350M down-shaped, n not a tile multiple
+    (2048, 2048, 5461, 512, 5464, {}),                   # 1B down-shaped, padded pitch
+    (1536, 4096, 1024, 1024, None, {}),                  # two row blocks of 512
+    (1024, 700, 640, 600, None, {}),                     # two row blocks of 320
+    (777, 320, 200, 320, None, {"identity": True}),      # dense gradient, idx = NULL
+    (64, 128, 128, 1, None, {}),                         # r = 1
+    (31, 64, 64, 64, None, {"with_rho": False}),         # fewer tokens than one block
+])
+def test_project_bf16_tensor_core(T, m, n, r, ldx, kw):
+    got, want = _project_case(T, m, n, r, torch.bfloat16, seed=T + n + r, ldx=ldx, **kw)
+    assert np.all(np.isfinite(got))
+    err = rel_fro(got, want)
+    assert err <= 1e-2                                    # acceptance tolerance
+    assert err <= 1e-4, err                               # what fp32 accumulation must deliver
+
+
+def test_project_bf16_is_bit_reproducible_and_flags_bad_rows():
+    T, m, n, r = 2048, 512, 512, 128
+    X = syn.make_X(T, n, torch.bfloat16).to(DEV)
+    dY = syn.make_dY(T, m, torch.bfloat16).to(DEV)
+    idx = torch.arange(0, 4 * r, 4, dtype=torch.int32, device=DEV)
+    ws = ws_bytes(grass.grass_project_workspace_bytes(T, m, n, r, grass.BF16))
+    outs = []
+    for _ in range(2):
+        Gc = torch.empty((r, n), dtype=torch.float32, device=DEV)
+        grass.grass_project_grad(dY, X, idx, None, r, Gc, ws)
+        grass.grass_device_status()
+        outs.append(Gc.clone())
+    assert torch.equal(outs[0], outs[1])
+    bad = idx.clone()
+    bad[5] = m + 3
+    Gc = torch.empty((r, n), dtype=torch.float32, device=DEV)
+    grass.grass_project_grad(dY, X, bad, None, r, Gc, ws)
+    status, detail = grass.grass_device_status(raise_on_error=False)
+    assert status == 1 and detail == m + 3
+    assert torch.all(Gc[5] == 0) and torch.equal(Gc[6], outs[0][6])
+
+
+# --------------------------------------------------------------------------- Adam
+@pytest.mark.parametrize("r,n,ld,step", [(32, 256, 256, 1), (128, 1376, 1376, 7), (5, 33, 40, 3),
+                                         (3, 8, 9, 1000)])
+def test_subspace_adam(r, n, ld, step):
+    g = torch.Generator().manual_seed(r + n)
+    Gc = torch.randn((r, n), generator=g) * torch.exp(2 * torch.randn((r, 1), generator=g))
+    M = torch.randn((r, n), generator=g) * 0.1 if step > 1 else torch.zeros((r, n))
+    V = torch.rand((r, n), generator=g) * 0.01 if step > 1 else torch.zeros((r, n))
+    lr, b1, b2, eps = 1e-3, 0.9, 0.999, 1e-8
+    Md, Vd = syn._padded(M.to(DEV), ld), syn._padded(V.to(DEV), ld)
+    Ud = syn._padded(torch.zeros((r, n), device=DEV), ld)
+    grass.grass_subspace_adam(Gc.to(DEV), Md, Vd, Ud, lr, b1, b2, eps, step)
+    grass.grass_device_status()
+    M1, V1, U1 = oracle.adam_update(f64(M), f64(V), f64(Gc), lr, b1, b2, eps, step)
+    # 1e-5 relative to the size of the terms that were added: M mixes two signed terms, so an
+    # element-wise bound relative to the (possibly cancelled) result would be ill-conditioned.
+    scale_M = b1 * np.abs(f64(M)) + (1 - b1) * np.abs(f64(Gc))
+    assert np.all(np.abs(f64(Md) - M1) <= 1e-5 * scale_M + 1e-30)
+    np.testing.assert_allclose(f64(Vd), V1, rtol=1e-5, atol=1e-30)
+    scale_U = lr * (scale_M / (1 - b1 ** step)) / (np.sqrt(V1 / (1 - b2 ** step)) + eps)
+    assert np.all(np.abs(f64(Ud) - U1) <= 1e-5 * scale_U + 1e-30)
+    assert rel_fro(f64(Md), M1) <= 1e-6 and rel_fro(f64(Ud), U1) <= 1e-6
+
+
+# --------------------------------------------------------------------------- scatter
+@pytest.mark.parametrize("m,n,ld,r,dtype", [
+    (256, 256, 256, 32, torch.float32), (512, 1376, 1376, 128, torch.bfloat16),
+    (100, 37, 40, 9, torch.bfloat16), (64, 5461, 5464, 16, torch.bfloat16),
+    (50, 30, 30, 50, torch.float32),
+])
+def test_scatter_update(m, n, ld, r, dtype):
+    rng = np.random.default_rng(m + n + r)
+    W = syn.make_W(m, n, dtype, seed0=r)
+    U = torch.tensor(rng.standard_normal((r, n)) * 1e-3, dtype=torch.float32)
+    sigma = np.sort(rng.choice(m, r, replace=True))
+    rho = (0.5 + 3 * rng.random(r)).astype(np.float32)
+    Wd = syn._padded(W.to(DEV), ld)
+    before = Wd.clone()
+    grass.grass_scatter_update(Wd, U.to(DEV), torch.tensor(sigma, dtype=torch.int32, device=DEV),
+                               torch.tensor(rho, device=DEV), 0.25)
+    grass.grass_device_status()
+    is_bf16 = dtype == torch.bfloat16
+    want = oracle.scatter_update(f64(W), f64(U), sigma, rho, 0.25, w_is_bf16=is_bf16)
+    got = f64(Wd)
+    untouched = np.setdiff1d(np.arange(m), sigma)
+    assert torch.equal(Wd[untouched], before[untouched])             # bit-identical
+    touched = np.unique(sigma)
+    if is_bf16:
+        exact = oracle.scatter_update(f64(W), f64(U), sigma, rho, 0.25)[touched]
+        ulp = np.ldexp(1.0, np.floor(np.log2(np.maximum(np.abs(exact), 2.0 ** -126))).astype(int) - 7)
+        diff = np.abs(got[touched] - want[touched])
+        assert np.all(diff <= ulp * 1.0001)
+        assert np.mean(diff > 0) < 0.01                              # rounding-boundary cases only
+    else:
+        np.testing.assert_allclose(got[touched], want[touched], rtol=1e-5, atol=1e-9)
+
+
+# --------------------------------------------------------------------------- whole step
+def _run_layer(m, n, T, r, dtype, method, K, steps, alpha, reset, seed, layer_id=0):
+    lr, b1, b2, eps = 1e-3, 0.9, 0.999, 1e-8
+    W = syn.make_W(m, n, dtype, seed0=seed)
+    batches = [(syn.make_dY(T, m, dtype, seed0=seed, step=t), syn.make_X(T, n, dtype, seed0=seed, step=t))
+               for t in range(steps)]
+    ws = grass.step.GrassWorkspace([(m, n)], T, r, dtype, method)
+    Wd = W.to(DEV).clone()
+    layer = grass.GrassLayer(Wd, r, method, K, alpha, lr, b1, b2, eps, reset_state=reset, seed=seed,
+                             layer_id=layer_id, workspace=ws)
+    trace = []
+    oracle.layer_steps(f64(W), [(f64(a), f64(b)) for a, b in batches], r, method, K, alpha, lr, b1,
+                       b2, eps, reset_state=reset, seed=seed, layer_id=layer_id,
+                       w_is_bf16=(dtype == torch.bfloat16), trace=trace)
+    for t, (dY, X) in enumerate(batches):
+        before = layer.W.clone()
+        layer.step(dY.to(DEV), X.to(DEV))
+        grass.grass_device_status()
+        ref = trace[t]
+        assert np.array_equal(layer.idx.cpu().numpy(), ref["sigma"]), f"step {t}: rows differ"
+        np.testing.assert_allclose(layer.rho.cpu().numpy(), ref["rho"], rtol=2e-5)
+        tol = 1e-5 if dtype == torch.float32 else 1e-4
+        assert rel_fro(f64(layer.Gc), ref["Gc"]) <= tol
+        assert rel_fro(f64(layer.M), ref["M"]) <= tol
+        assert rel_fro(f64(layer.V), ref["V"]) <= 2 * tol
+        assert rel_fro(f64(layer.U), ref["U"]) <= 10 * tol
+        untouched = np.setdiff1d(np.arange(m), ref["sigma"])
+        got = f64(layer.W)
+        assert torch.equal(layer.W[untouched], before[untouched])      # bit-identical
+        if dtype == torch.float32:
+            np.testing.assert_allclose(got, ref["W"], rtol=1e-5, atol=1e-8)
+        else:
+            assert np.max(np.abs(got - ref["W"])) <= 2.0 ** -7 * np.max(np.abs(ref["W"]))
+            assert np.mean(got != ref["W"]) < 0.02
+    return layer
+
+
+def test_layer_steps_config1_fp32_topr():
+    """m = n = 256, T = 512, r = 32, top-r, K = 1, 3 steps, fp32 everywhere, seed 0."""
+    _run_layer(256, 256, 512, 32, torch.float32, grass.SEL_TOPR, K=1, steps=3, alpha=1.0,
+               reset=True, seed=0)
+
+
+def test_layer_steps_bf16_multinomial_with_refresh():
+    """60M-shaped q projection at reduced T: multinomial-norm, rho, refresh at t = 0 and 2."""
+    _run_layer(512, 512, 2048, 128, torch.bfloat16, grass.SEL_MULTINOMIAL_NORM, K=2, steps=4,
+               alpha=0.25, reset=False, seed=3, layer_id=5)
+
+
+def test_layer_steps_bf16_topr_reset():
+    _run_layer(1376, 512, 1024, 128, torch.bfloat16, grass.SEL_TOPR, K=2, steps=3, alpha=0.25,
+               reset=True, seed=4)
