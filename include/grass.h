@@ -13,8 +13,8 @@
  * Conventions shared by every call
  *   - Every pointer is a DEVICE pointer unless it is marked "host".  The caller
  *     owns all buffers; the library allocates no device memory and keeps no
- *     state between calls except an encoded-descriptor cache on the host and one
- *     small per-device status word (see grass_device_status).
+ *     state between calls except one small per-device status word (see
+ *     grass_device_status).
  *   - Matrices are row-major; a leading dimension `ld*` is the row pitch in
  *     ELEMENTS and must be >= the row length.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
@@ -156,6 +156,31 @@ int grass_scatter_update(void* W, int wdt, int64_t m, int64_t n, int64_t ldw, co
 int grass_device_status(void* stream, int32_t* detail);
 
 const char* grass_status_string(int status);
+
+/*
+ * Per-launch timing of the library's own kernels (a measurement aid; the paper
+ * has no counterpart).  Between grass_profile_begin and grass_profile_end every
+ * kernel the library launches on the calling thread's behalf is bracketed by a
+ * pair of CUDA events recorded on the launch stream, up to max_launches
+ * launches (later ones are counted but not timed).  grass_profile_end
+ * synchronises the device, writes for launch i its kernel id (grass_kernel_t)
+ * and duration in milliseconds to the HOST arrays kernel_id[i] and ms[i]
+ * (each of capacity max_launches; either may be NULL), returns the number of
+ * launches seen in *n_launches (host) and releases the events.  Not
+ * thread-safe; one profile at a time per process.
+ */
+typedef enum {
+  GRASS_K_ROW_NORMS = 0,
+  GRASS_K_SELECT = 1,
+  GRASS_K_GATHER = 2,        /* copy of the selected dY columns */
+  GRASS_K_PROJECT_TC = 3,    /* tcgen05 projection GEMM */
+  GRASS_K_SPLITK_REDUCE = 4,
+  GRASS_K_PROJECT_FP32 = 5,
+  GRASS_K_ADAM = 6,
+  GRASS_K_SCATTER = 7
+} grass_kernel_t;
+int grass_profile_begin(int32_t max_launches);
+int grass_profile_end(int32_t* kernel_id, float* ms, int32_t* n_launches);
 
 #ifdef __cplusplus
 }

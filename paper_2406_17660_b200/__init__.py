@@ -10,6 +10,6 @@ from .binding import (  # noqa: F401
     grass_row_norms, grass_select, grass_select_workspace_bytes,
     grass_project_grad, grass_project_workspace_bytes,
     grass_subspace_adam, grass_scatter_update, grass_device_status,
-    grass_status_string, library_path, load_library,
+    grass_status_string, grass_profile_begin, grass_profile_end, library_path, load_library,
 )
 from .step import GrassLayer  # noqa: F401

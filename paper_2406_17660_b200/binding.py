@@ -44,7 +44,13 @@ _SIGNATURES = {
                                      c_void_p, c_void_p, c_int32, c_double, c_void_p]),
     "grass_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int32)]),
     "grass_status_string": (ctypes.c_char_p, [c_int]),
+    "grass_profile_begin": (c_int, [c_int32]),
+    "grass_profile_end": (c_int, [ctypes.POINTER(c_int32), ctypes.POINTER(ctypes.c_float),
+                                  ctypes.POINTER(c_int32)]),
 }
+
+KERNEL_NAMES = ["row_norms", "select", "gather", "project_tc", "splitk_reduce", "project_fp32",
+                "adam", "scatter"]
 
 
 def load_library():
@@ -175,3 +181,19 @@ def grass_device_status(raise_on_error: bool = True):
     if status != 0 and raise_on_error:
         raise GrassError(status, f"device status (detail {detail.value})")
     return status, detail.value
+
+
+def grass_profile_begin(max_launches: int) -> None:
+    _check(load_library().grass_profile_begin(max_launches), "grass_profile_begin")
+    grass_profile_begin.cap = max_launches
+
+
+def grass_profile_end():
+    """Returns (launches_seen, [(kernel_name, ms), ...]) for the launches that were timed."""
+    cap = grass_profile_begin.cap
+    kid = (c_int32 * cap)()
+    ms = (ctypes.c_float * cap)()
+    n = c_int32(0)
+    _check(load_library().grass_profile_end(kid, ms, ctypes.byref(n)), "grass_profile_end")
+    timed = min(n.value, cap)
+    return n.value, [(KERNEL_NAMES[kid[i]], float(ms[i])) for i in range(timed)]

@@ -94,6 +94,7 @@ extern "C" int grass_subspace_adam(const float* Gc, int64_t ldgc, float* M, floa
   const bool vec = (n % 4 == 0) && (ldgc % 4 == 0) && (ldstate % 4 == 0) && aligned_to(Gc, 16) &&
                    aligned_to(M, 16) && aligned_to(V, 16) && aligned_to(U, 16);
   const int64_t max_blocks = 148LL * 16;
+  ProfileScope prof(GRASS_K_ADAM, s);
   if (vec) {
     const int64_t nv = n / 4, total = static_cast<int64_t>(r) * nv;
     int64_t blocks = (total + kThreads - 1) / kThreads;

@@ -19,6 +19,15 @@ __device__ __forceinline__ void record_status(int* status, int code, int detail)
 // Device address of the current device's status word (host function, common.cu).
 int* status_word(cudaError_t* err);
 
+// Brackets one kernel launch with events while a profile is active (common.cu).
+void profile_mark_begin(int kernel_id, cudaStream_t s);
+void profile_mark_end(cudaStream_t s);
+struct ProfileScope {
+  cudaStream_t s;
+  ProfileScope(int kernel_id, cudaStream_t stream) : s(stream) { profile_mark_begin(kernel_id, s); }
+  ~ProfileScope() { profile_mark_end(s); }
+};
+
 #define GRASS_CUDA_TRY(expr)                                                             \
   do {                                                                                   \
     cudaError_t e__ = (expr);                                                            \

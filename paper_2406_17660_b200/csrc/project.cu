@@ -138,9 +138,12 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
     __nv_bfloat16* Ag = reinterpret_cast<__nv_bfloat16*>(wsp);
     dim3 ggrid(static_cast<unsigned>((plan.r_pad / 8 + kGatherThreads - 1) / kGatherThreads),
                static_cast<unsigned>((T + kGatherTokens - 1) / kGatherTokens));
-    gather_cols_kernel<<<ggrid, kGatherThreads, 0, s>>>(
-        static_cast<const __nv_bfloat16*>(dY), lddy, static_cast<int>(T), static_cast<int>(m), idx,
-        r, plan.r_pad, Ag, status);
+    {
+      ProfileScope prof(GRASS_K_GATHER, s);
+      gather_cols_kernel<<<ggrid, kGatherThreads, 0, s>>>(
+          static_cast<const __nv_bfloat16*>(dY), lddy, static_cast<int>(T), static_cast<int>(m),
+          idx, r, plan.r_pad, Ag, status);
+    }
     GRASS_LAUNCH_CHECK();
     if (!make_map(&tmA, Ag, T, plan.r_pad, plan.r_pad)) return GRASS_ERR_CUDA;
     wsp += plan.ag_bytes;
@@ -171,13 +174,17 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   }
   dim3 grid(static_cast<unsigned>(plan.n_blocks), static_cast<unsigned>(plan.r_blocks),
             static_cast<unsigned>(plan.split_k));
-  project_tc_kernel<<<grid, kTcThreads, plan.smem_bytes, s>>>(tmX, tmA, p);
+  {
+    ProfileScope prof(GRASS_K_PROJECT_TC, s);
+    project_tc_kernel<<<grid, kTcThreads, plan.smem_bytes, s>>>(tmX, tmA, p);
+  }
   GRASS_LAUNCH_CHECK();
   if (plan.split_k > 1) {
     const int vec = (n % 4 == 0) && (ldgc % 4 == 0) && aligned_to(Gc, 16);
     const long long work = static_cast<long long>(r) * (vec ? n / 4 : n);
     long long blocks = (work + 255) / 256;
     if (blocks > kSmCount * 8) blocks = kSmCount * 8;
+    ProfileScope prof(GRASS_K_SPLITK_REDUCE, s);
     splitk_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(
         p.out, plan.ld_part, p.split_stride, plan.split_k, r, static_cast<int>(n), rho, Gc, ldgc,
         vec);
@@ -218,6 +225,7 @@ extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, i
   if (status == nullptr) GRASS_CUDA_TRY(err);
   dim3 grid(static_cast<unsigned>((n + kSimtBC - 1) / kSimtBC),
             static_cast<unsigned>((r + kSimtBJ - 1) / kSimtBJ));
+  ProfileScope prof(GRASS_K_PROJECT_FP32, s);
   project_simt_kernel<float><<<grid, kSimtThreads, 0, s>>>(
       static_cast<const float*>(dY), lddy, static_cast<const float*>(X), ldx, T, m, n, idx, rho, r,
       Gc, ldgc, status);

@@ -91,6 +91,7 @@ int launch(const void* G, int64_t m, int64_t n, int64_t ldg, float* norms, cudaS
   const T* g = static_cast<const T*>(G);
   const bool vec = aligned_to(G, 16) && (ldg % Vec<T>::N) == 0;
   const bool wide = n > 2048;  // long rows: one CTA per row
+  ProfileScope prof(GRASS_K_ROW_NORMS, s);
   if (wide) {
     const unsigned grid = static_cast<unsigned>(m);
     if (vec) row_norms_kernel<T, kThreads, true><<<grid, kThreads, 0, s>>>(g, m, n, ldg, norms);

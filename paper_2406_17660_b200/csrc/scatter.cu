@@ -98,6 +98,7 @@ int launch(void* W, int64_t m, int64_t n, int64_t ldw, const float* U, int64_t l
                    aligned_to(U, 16);
   dim3 grid(static_cast<unsigned>((n + kThreads * N - 1) / (kThreads * N)),
             static_cast<unsigned>(r));
+  ProfileScope prof(GRASS_K_SCATTER, s);
   if (vec)
     scatter_kernel<T, true><<<grid, kThreads, 0, s>>>(static_cast<T*>(W), m, n, ldw, U, ldu, idx,
                                                       rho, r, alpha, status);

@@ -258,7 +258,10 @@ extern "C" int grass_select(const float* norms, int64_t m, int32_t r, int method
   a.epoch = epoch;
   a.idx = idx;
   a.rho = rho;
-  select_kernel<<<1, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  {
+    ProfileScope prof(GRASS_K_SELECT, static_cast<cudaStream_t>(stream));
+    select_kernel<<<1, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  }
   GRASS_LAUNCH_CHECK();
   return GRASS_OK;
 }
