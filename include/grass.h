@@ -93,6 +93,37 @@ int grass_select(const float* norms, int64_t m, int32_t r, int method, uint64_t 
                  size_t ws_bytes, void* stream);
 
 /*
+ * grass_select without a workspace argument, for callers that cannot obtain
+ * device memory at the point of the call (the paper has no counterpart; it is
+ * a packaging variant of the call above and computes exactly the same idx and
+ * rho).  Typical callers: an optimizer hook running inside a framework whose
+ * pooling allocator already owns the whole device, so that a raw cudaMalloc
+ * would fail; a plugin that is handed tensors but no allocator; a step on a
+ * latency-critical path where the device-wide synchronisation an allocation
+ * implies is not acceptable.  The scratch (the fp64 running sum and the
+ * per-row hit counters) lives in a fixed array inside the library image:
+ * GRASS_SELECT_STATIC_MAX_M rows, 12 bytes each (192 KiB), held by every GPU
+ * that loads the library until the process exits.
+ *   - m > GRASS_SELECT_STATIC_MAX_M returns GRASS_ERR_WORKSPACE (and says so on
+ *     stderr); nothing is launched.  All other arguments and errors are as for
+ *     grass_select.
+ *   - The call allocates nothing, on the host or the device.  The first call
+ *     on each device looks up the array's device address (with that device
+ *     current) and caches it; make that first call during start-up, outside
+ *     any stream capture.
+ *   - All calls on a device share the one array, which still holds what the
+ *     previous call left there.  The kernel overwrites or zeroes every entry
+ *     before reading it, so calls that follow one another on a stream are
+ *     independent; two calls that may run at the same time on one GPU (two
+ *     streams, two host threads) race on the array and must be serialised by
+ *     the caller.
+ */
+#define GRASS_SELECT_STATIC_MAX_M 16384
+int grass_select_static(const float* norms, int64_t m, int32_t r, int method, uint64_t seed,
+                        uint32_t layer_id, uint32_t epoch, int32_t* idx, float* rho,
+                        void* stream);
+
+/*
  * Projected gradient (Section 3.1, "Efficient Gradient Projection"):
  *   Gc[j, c] = rho_j * sum_t dY[t, idx_j] * X[t, c],   j < r, c < n,
  * i.e. rho ((B dY^T) X); the m x n gradient is never formed.

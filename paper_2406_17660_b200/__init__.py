@@ -7,7 +7,7 @@ raises if it has not been built.
 """
 from .binding import (  # noqa: F401
     GrassError, BF16, F32, SEL_TOPR, SEL_MULTINOMIAL_NORM,
-    grass_row_norms, grass_select, grass_select_workspace_bytes,
+    grass_row_norms, grass_select, grass_select_static, grass_select_workspace_bytes,
     grass_project_grad, grass_project_workspace_bytes,
     grass_subspace_adam, grass_scatter_update, grass_device_status,
     grass_status_string, grass_profile_begin, grass_profile_end, library_path, load_library,

@@ -33,6 +33,8 @@ _SIGNATURES = {
     "grass_select_workspace_bytes": (c_size_t, [c_int64, c_int32, c_int]),
     "grass_select": (c_int, [c_void_p, c_int64, c_int32, c_int, c_uint64, c_uint32, c_uint32,
                              c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "grass_select_static": (c_int, [c_void_p, c_int64, c_int32, c_int, c_uint64, c_uint32, c_uint32,
+                                    c_void_p, c_void_p, c_void_p]),
     "grass_project_workspace_bytes": (c_size_t, [c_int64, c_int64, c_int64, c_int32, c_int]),
     "grass_project_grad": (c_int, [c_void_p, c_int64, c_void_p, c_int64, c_int, c_int64, c_int64,
                                    c_int64, c_void_p, c_void_p, c_int32, c_void_p, c_int64,
@@ -129,6 +131,18 @@ def grass_select(norms, r, method, seed, layer_id, epoch, idx, rho, ws) -> None:
     _check(load_library().grass_select(_ptr(norms), norms.numel(), r, method, seed, layer_id, epoch,
                                        _ptr(idx), _ptr(rho), _ptr(ws), ws_bytes, _stream()),
            "grass_select")
+
+
+def grass_select_static(norms, r, method, seed, layer_id, epoch, idx, rho) -> None:
+    """grass_select with the library's built-in scratch: no workspace argument, nothing is
+    allocated.  For callers that have tensors but no way to get device memory at this point
+    (see include/grass.h for the size limit and the sharing rules)."""
+    _require(norms, torch.float32, "norms")
+    _require(idx, torch.int32, "idx")
+    _require(rho, torch.float32, "rho")
+    _check(load_library().grass_select_static(_ptr(norms), norms.numel(), r, method, seed, layer_id,
+                                              epoch, _ptr(idx), _ptr(rho), _stream()),
+           "grass_select_static")
 
 
 def grass_project_workspace_bytes(T: int, m: int, n: int, r: int, dt: int) -> int:

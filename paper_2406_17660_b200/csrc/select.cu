@@ -265,3 +265,77 @@ extern "C" int grass_select(const float* norms, int64_t m, int32_t r, int method
   GRASS_LAUNCH_CHECK();
   return GRASS_OK;
 }
+
+// ---------------------------------------------------------------------------
+// grass_select_static: the same selection with its scratch in a fixed device
+// array that is part of the library image, for callers that cannot allocate.
+// ---------------------------------------------------------------------------
+namespace grass {
+namespace {
+
+constexpr int kStaticMaxM = GRASS_SELECT_STATIC_MAX_M;
+
+// Running sum (fp64) followed by the per-row hit counts (int32) for up to
+// kStaticMaxM rows: 192 KiB, resident on every GPU that loads the library.
+static __device__ __align__(256) unsigned char g_select_scratch[kStaticMaxM * (sizeof(double) + sizeof(int))];
+
+// Device address of g_select_scratch on the current device, resolved once per
+// device.  In host code the symbol name is only a handle; a kernel must be
+// given the address the runtime reports for it.
+int static_scratch(unsigned char** out) {
+  static unsigned char* cached[64] = {nullptr};
+  int dev = 0;
+  GRASS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return GRASS_ERR_INVALID_ARG;
+  if (cached[dev] == nullptr) {
+    unsigned char* p = nullptr;
+    GRASS_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_select_scratch));
+    cached[dev] = p;
+  }
+  *out = cached[dev];
+  return GRASS_OK;
+}
+
+}  // namespace
+}  // namespace grass
+
+extern "C" int grass_select_static(const float* norms, int64_t m, int32_t r, int method,
+                                   uint64_t seed, uint32_t layer_id, uint32_t epoch, int32_t* idx,
+                                   float* rho, void* stream) {
+  using namespace grass;
+  if (norms == nullptr || idx == nullptr || rho == nullptr || m < 1 || r < 1 || r > m)
+    return GRASS_ERR_INVALID_ARG;
+  if (m > kStaticMaxM) {
+    fprintf(stderr, "grass_select_static: m = %lld exceeds the built-in scratch (%d rows); "
+                    "use grass_select with a caller-provided workspace\n",
+            static_cast<long long>(m), kStaticMaxM);
+    return GRASS_ERR_WORKSPACE;
+  }
+  if (method != GRASS_SEL_TOPR && method != GRASS_SEL_MULTINOMIAL_NORM)
+    return GRASS_ERR_UNSUPPORTED;
+  unsigned char* scratch = nullptr;
+  const int rc = static_scratch(&scratch);
+  if (rc != GRASS_OK) return rc;
+  cudaError_t err;
+  SelectArgs a;
+  a.status = status_word(&err);
+  if (a.status == nullptr) GRASS_CUDA_TRY(err);
+  a.cdf = reinterpret_cast<double*>(scratch);
+  a.counts = reinterpret_cast<int*>(scratch + static_cast<size_t>(kStaticMaxM) * sizeof(double));
+  a.norms = norms;
+  a.m = static_cast<int>(m);
+  a.r = r;
+  a.method = method;
+  a.seed_lo = static_cast<uint32_t>(seed & 0xffffffffu);
+  a.seed_hi = static_cast<uint32_t>(seed >> 32);
+  a.layer_id = layer_id;
+  a.epoch = epoch;
+  a.idx = idx;
+  a.rho = rho;
+  // The kernel writes every running-sum entry it later reads and zeroes the
+  // m hit counters before counting, so whatever an earlier call left in the
+  // array is never observed.
+  select_kernel<<<1, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  GRASS_LAUNCH_CHECK();
+  return GRASS_OK;
+}
