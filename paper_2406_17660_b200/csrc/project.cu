@@ -2,6 +2,7 @@
 // launches).  The kernels are in project_tc.cuh (bf16, tcgen05) and
 // project_simt.cuh (fp32).
 #include <cudaTypedefs.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "project_simt.cuh"
@@ -11,7 +12,6 @@ namespace grass {
 namespace {
 
 constexpr int kSmCount = 148;
-constexpr size_t kSmemBudget = 227 * 1024 - 1024;  // dynamic part; the rest holds the barriers
 
 struct TcPlan {
   int r_pad;      // r_blocks * r_cta: width of the gathered operand
@@ -65,10 +65,8 @@ TcPlan make_plan(int64_t T, int64_t n, int r) {
     }
   }
   p.n_blocks = static_cast<int>((n + p.MB * 128 - 1) / (p.MB * 128));
-  const size_t stage_bytes = static_cast<size_t>(2 * p.MB + p.r_cta / 64) * kTcSlabBytes;
-  const int stages = static_cast<int>((kSmemBudget - 1024) / stage_bytes);
-  p.stages = stages > kTcMaxStages ? kTcMaxStages : stages;
-  p.smem_bytes = p.stages * stage_bytes + 1024;
+  p.stages = tc_stages(p.MB, p.r_cta / 64);
+  p.smem_bytes = static_cast<size_t>(p.stages) * tc_stage_bytes(p.MB, p.r_cta / 64) + 1024;
   p.ld_part = static_cast<long long>(round_up(static_cast<size_t>(n), 4));
   p.ag_bytes = round_up(static_cast<size_t>(T) * p.r_pad * sizeof(__nv_bfloat16), 256);
   p.part_bytes = p.split_k > 1
@@ -107,6 +105,39 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
   return true;
 }
 
+template <int MB, int NSLAB>
+int launch_tc_one(dim3 grid, size_t smem, cudaStream_t s, const CUtensorMap& tmX,
+                  const CUtensorMap& tmA, const TcParams& p) {
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  GRASS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel<MB, NSLAB>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kTcSmemBudget));
+    attr_set[dev] = true;
+  }
+  {
+    ProfileScope prof(GRASS_K_PROJECT_TC, s);
+    project_tc_kernel<MB, NSLAB><<<grid, kTcThreads, smem, s>>>(tmX, tmA, p);
+  }
+  GRASS_LAUNCH_CHECK();
+  return GRASS_OK;
+}
+
+// (MB, NSLAB) with MB * 64 * NSLAB <= 512 TMEM columns.
+int launch_tc(int MB, int nslab, dim3 grid, size_t smem, cudaStream_t s, const CUtensorMap& tmX,
+              const CUtensorMap& tmA, const TcParams& p) {
+#define GRASS_TC_CASE(mb, ns) \
+  if (MB == mb && nslab == ns) return launch_tc_one<mb, ns>(grid, smem, s, tmX, tmA, p)
+  GRASS_TC_CASE(1, 1); GRASS_TC_CASE(1, 2); GRASS_TC_CASE(1, 3); GRASS_TC_CASE(1, 4);
+  GRASS_TC_CASE(1, 5); GRASS_TC_CASE(1, 6); GRASS_TC_CASE(1, 7); GRASS_TC_CASE(1, 8);
+  GRASS_TC_CASE(2, 1); GRASS_TC_CASE(2, 2); GRASS_TC_CASE(2, 3); GRASS_TC_CASE(2, 4);
+  GRASS_TC_CASE(4, 1); GRASS_TC_CASE(4, 2);
+#undef GRASS_TC_CASE
+  return GRASS_ERR_UNSUPPORTED;
+}
+
 int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T, int64_t m,
                  int64_t n, const int32_t* idx, const float* rho, int r, float* Gc, int64_t ldgc,
                  void* ws, size_t ws_bytes, cudaStream_t s) {
@@ -120,16 +151,6 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   cudaError_t err;
   int* status = status_word(&err);
   if (status == nullptr) GRASS_CUDA_TRY(err);
-
-  static bool attr_set[64] = {false};
-  int dev = 0;
-  GRASS_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        static_cast<int>(kSmemBudget)));
-    attr_set[dev] = true;
-  }
 
   char* wsp = static_cast<char*>(ws);
   CUtensorMap tmX, tmA;
@@ -155,12 +176,13 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   p.T = static_cast<int>(T);
   p.n = static_cast<int>(n);
   p.r = r;
-  p.r_cta = plan.r_cta;
-  p.MB = plan.MB;
-  p.stages = plan.stages;
   p.k_blocks = plan.k_blocks;
   p.split_k = plan.split_k;
   p.status = status;
+  if (getenv("GRASS_DEBUG_PLAN") != nullptr)
+    fprintf(stderr, "grass plan T=%lld n=%lld r=%d: r_cta=%d r_blocks=%d MB=%d n_blocks=%d "
+                    "split_k=%d stages=%d\n", static_cast<long long>(T), static_cast<long long>(n),
+            r, plan.r_cta, plan.r_blocks, plan.MB, plan.n_blocks, plan.split_k, plan.stages);
   if (plan.split_k == 1) {
     p.out = Gc;
     p.ld_out = ldgc;
@@ -174,11 +196,8 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   }
   dim3 grid(static_cast<unsigned>(plan.n_blocks), static_cast<unsigned>(plan.r_blocks),
             static_cast<unsigned>(plan.split_k));
-  {
-    ProfileScope prof(GRASS_K_PROJECT_TC, s);
-    project_tc_kernel<<<grid, kTcThreads, plan.smem_bytes, s>>>(tmX, tmA, p);
-  }
-  GRASS_LAUNCH_CHECK();
+  const int rc = launch_tc(plan.MB, plan.r_cta / 64, grid, plan.smem_bytes, s, tmX, tmA, p);
+  if (rc != GRASS_OK) return rc;
   if (plan.split_k > 1) {
     const int vec = (n % 4 == 0) && (ldgc % 4 == 0) && aligned_to(Gc, 16);
     const long long work = static_cast<long long>(r) * (vec ? n / 4 : n);

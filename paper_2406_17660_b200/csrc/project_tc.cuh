@@ -3,9 +3,9 @@
 //
 // The contraction runs over tokens (T = 32K..64K) while the output r x n is
 // small, so the kernel is organised around one rule: read X once.  A CTA owns
-// an output tile of (MB * 128) columns of n by r_cta selected rows with
-// MB * r_cta <= 512, i.e. all 512 fp32 TMEM columns, and a slice of the tokens
-// (split-K); every X element it loads meets all r_cta rows.
+// an output tile of (MB * 128) columns of n by r_cta = 64 * NSLAB selected rows
+// with MB * r_cta <= 512, i.e. up to all 512 fp32 TMEM columns, and a slice of
+// the tokens (split-K); every X element it loads meets all r_cta rows.
 //
 // Operand roles are swapped with respect to the formula so that neither input
 // needs a transpose in HBM:  D^T[c, j] = sum_t X[t, c] * A[t, j]  with
@@ -16,8 +16,14 @@
 // column = j, so the epilogue's tcgen05.ld hands each warp 32 consecutive c for
 // one j per register: every store instruction writes 128 contiguous bytes.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA
-// issuer, warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4)..+31).
+// Warp roles (320 threads): warp 0 = TMA producer (one lane per slab), warp 1 =
+// TMEM owner + single-thread MMA issuer, warps 2..9 = epilogue (warp w reads
+// TMEM lanes 32*(w%4)..+31; the two warps of a lane quarter alternate over the
+// 32-column chunks).  A lone issuing thread retires roughly one dependent
+// instruction every 4-5 clocks, so the per-stage instruction count of the
+// producer and of the MMA issuer bounds the pipeline: tile shape and stage
+// count are template parameters so that every descriptor is a constant plus
+// the stage offset and the loops unroll.
 // Every mbarrier wait is bounded; on expiry the CTA records GRASS_ERR_TIMEOUT,
 // drains what it has in flight (bounded again), frees its TMEM and returns.
 #pragma once
@@ -29,16 +35,21 @@ namespace grass {
 
 constexpr int kTcBK = 32;                 // tokens per pipeline stage
 constexpr int kTcSlabBytes = kTcBK * 128; // [32 tokens][64 bf16]
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 320;
 constexpr int kTcMaxStages = 8;
+constexpr int kTcSmemBudget = 227 * 1024 - 1024;  // dynamic part; the rest holds the barriers
 constexpr long long kTcWaitLimit = 2000000000LL;  // SM clocks (~1 s)
 constexpr long long kTcDrainLimit = 200000000LL;  // give-up path: wait for work in flight
 
+__host__ __device__ constexpr int tc_stage_bytes(int MB, int NSLAB) { return (2 * MB + NSLAB) * kTcSlabBytes; }
+__host__ __device__ constexpr int tc_stages(int MB, int NSLAB) {
+  return (kTcSmemBudget - 1024) / tc_stage_bytes(MB, NSLAB) > kTcMaxStages
+             ? kTcMaxStages
+             : (kTcSmemBudget - 1024) / tc_stage_bytes(MB, NSLAB);
+}
+
 struct TcParams {
   int T, n, r;          // logical sizes
-  int r_cta;            // selected rows per CTA, multiple of 64, <= 512
-  int MB;               // 128-column blocks of n per CTA: 1, 2 or 4; MB * r_cta <= 512
-  int stages;           // pipeline depth
   int k_blocks;         // ceil(T / 32)
   int split_k;          // gridDim.z
   float* out;           // split_k == 1: Gc, else partials [split][r][ld_out]
@@ -48,9 +59,18 @@ struct TcParams {
   int* status;
 };
 
+template <int MB, int NSLAB>
 __global__ void __launch_bounds__(kTcThreads, 1)
 project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA,
                   const TcParams p) {
+  constexpr int R_CTA = 64 * NSLAB;
+  constexpr int X_SLABS = 2 * MB;
+  constexpr int N_SLABS = X_SLABS + NSLAB;
+  constexpr int STAGE_BYTES = tc_stage_bytes(MB, NSLAB);
+  constexpr int STAGES = tc_stages(MB, NSLAB);
+  static_assert(MB * R_CTA <= 512, "accumulators exceed TMEM");
+  static_assert(N_SLABS <= 32, "one producer lane per slab");
+
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kTcMaxStages];
   __shared__ __align__(8) uint64_t bar_empty[kTcMaxStages];
@@ -61,12 +81,9 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                               ~static_cast<uintptr_t>(1023));
-  const int x_slabs = 2 * p.MB, a_slabs = p.r_cta / 64;
-  const uint32_t stage_bytes = static_cast<uint32_t>((x_slabs + a_slabs) * kTcSlabBytes);
-
-  const int c_tile0 = blockIdx.x * p.MB * 128;
-  const int r0 = blockIdx.y * p.r_cta;
-  // this CTA's token blocks: [kb_begin, kb_end)
+  const int c_tile0 = blockIdx.x * (MB * 128);
+  const int r0 = blockIdx.y * R_CTA;
+  // this CTA's token blocks: [kb_begin, kb_begin + kb_count)
   const int kb_per = p.k_blocks / p.split_k, kb_rem = p.k_blocks % p.split_k;
   const int z = blockIdx.z;
   const int kb_begin = z * kb_per + (z < kb_rem ? z : kb_rem);
@@ -74,7 +91,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 
   if (threadIdx.x == 0) {
     s_abort = 0;
-    for (int s = 0; s < p.stages; ++s) {
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) {
       ptx::mbar_init(&bar_full[s], 1);
       ptx::mbar_init(&bar_empty[s], 1);
     }
@@ -94,45 +112,48 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   volatile int* abort_flag = &s_abort;
 
   if (warp == 0) {
-    // ================= TMA producer =================
-    if (lane == 0) {
-      int issued = 0;
-      for (int it = 0; it < kb_count; ++it) {
-        const int s = it % p.stages;
-        const uint32_t ph = static_cast<uint32_t>(it / p.stages) & 1u;
-        if (!ptx::mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kTcWaitLimit)) {
+    // ================= TMA producer: one lane per slab =================
+    const bool is_x = lane < X_SLABS;
+    const CUtensorMap* map = is_x ? &tmX : &tmA;
+    const int xcoord = is_x ? c_tile0 + lane * 64 : r0 + (lane - X_SLABS) * 64;
+    uint8_t* my_dst = tiles + lane * kTcSlabBytes;
+    int tok = kb_begin * kTcBK;
+    int s = 0, issued = 0;
+    uint32_t ph = 0;
+    for (int it = 0; it < kb_count; ++it) {
+      int ok = 1;
+      if (lane == 0) {
+        ok = ptx::mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kTcWaitLimit) ? 1 : 0;
+        if (ok) {
+          ptx::mbar_arrive_expect_tx(&bar_full[s], STAGE_BYTES);
+        } else {
           if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 100 + s);
           *abort_flag = 1;
-          break;
         }
-        ptx::mbar_arrive_expect_tx(&bar_full[s], stage_bytes);
-        uint8_t* dst = tiles + static_cast<size_t>(s) * stage_bytes;
-        const int tok = (kb_begin + it) * kTcBK;
-        for (int i = 0; i < x_slabs; ++i)
-          ptx::tma_load_2d(dst + i * kTcSlabBytes, &tmX, c_tile0 + i * 64, tok, &bar_full[s]);
-        dst += x_slabs * kTcSlabBytes;
-        for (int i = 0; i < a_slabs; ++i)
-          ptx::tma_load_2d(dst + i * kTcSlabBytes, &tmA, r0 + i * 64, tok, &bar_full[s]);
-        issued = it + 1;
       }
-      if (*abort_flag != 0) {
-        // let the copies already issued land before the CTA gives its smem back
-        const int first = issued > p.stages ? issued - p.stages : 0;
-        for (int it = first; it < issued; ++it)
-          ptx::mbar_wait_bounded(&bar_full[it % p.stages],
-                                 static_cast<uint32_t>(it / p.stages) & 1u, nullptr,
-                                 kTcDrainLimit);
-      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane < N_SLABS) ptx::tma_load_2d(my_dst + s * STAGE_BYTES, map, xcoord, tok, &bar_full[s]);
+      tok += kTcBK;
+      issued = it + 1;
+      if (++s == STAGES) { s = 0; ph ^= 1u; }
+    }
+    if (lane == 0 && *abort_flag != 0) {
+      // let the copies already issued land before the CTA gives its smem back
+      const int first = issued > STAGES ? issued - STAGES : 0;
+      for (int it = first; it < issued; ++it)
+        ptx::mbar_wait_bounded(&bar_full[it % STAGES], static_cast<uint32_t>(it / STAGES) & 1u,
+                               nullptr, kTcDrainLimit);
     }
   } else if (warp == 1) {
-    // ================= MMA issuer =================
+    // ================= MMA issuer: one thread =================
     if (lane == 0) {
-      const uint32_t tiles_addr = ptx::smem_u32(tiles);
-      const uint32_t lbo = kTcSlabBytes, sbo = 1024;
+      constexpr uint32_t LBO = kTcSlabBytes, SBO = 1024;
+      const uint64_t desc0 = ptx::smem_desc_mn_sw128(ptx::smem_u32(tiles), LBO, SBO);
       bool ok = true;
-      for (int it = 0; it < kb_count && ok; ++it) {
-        const int s = it % p.stages;
-        const uint32_t ph = static_cast<uint32_t>(it / p.stages) & 1u;
+      int s = 0;
+      uint32_t ph = 0;
+      for (int it = 0; it < kb_count; ++it) {
         if (!ptx::mbar_wait_bounded(&bar_full[s], ph, abort_flag, kTcWaitLimit)) {
           if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 200 + s);
           *abort_flag = 1;
@@ -140,59 +161,79 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           break;
         }
         ptx::fence_tc_after_sync();
-        const uint32_t xs = tiles_addr + static_cast<uint32_t>(s) * stage_bytes;
-        const uint32_t as = xs + static_cast<uint32_t>(x_slabs * kTcSlabBytes);
+        const uint64_t dstage = desc0 + static_cast<uint64_t>((s * STAGE_BYTES) >> 4);
 #pragma unroll
         for (int ks = 0; ks < kTcBK / 16; ++ks) {
-          const uint32_t koff = static_cast<uint32_t>(ks) * 2u * sbo;  // 16 tokens = 2 groups of 8
-          const uint32_t acc = (it > 0 || ks > 0) ? 1u : 0u;
-          for (int mb = 0; mb < p.MB; ++mb) {
-            const uint64_t adesc = ptx::smem_desc_mn_sw128(
-                xs + static_cast<uint32_t>(mb * 2 * kTcSlabBytes) + koff, lbo, sbo);
-            for (int j = 0; j < p.r_cta; j += 256) {
-              const int ncols = p.r_cta - j < 256 ? p.r_cta - j : 256;
-              const uint64_t bdesc = ptx::smem_desc_mn_sw128(
-                  as + static_cast<uint32_t>((j / 64) * kTcSlabBytes) + koff, lbo, sbo);
-              ptx::mma_bf16(tmem_base + static_cast<uint32_t>(mb * p.r_cta + j), adesc, bdesc,
+          const uint32_t acc = (it | ks) != 0 ? 1u : 0u;
+#pragma unroll
+          for (int mb = 0; mb < MB; ++mb) {
+            // 16 tokens = 2 groups of 8 rows = 2 * SBO bytes into every slab
+            const uint64_t adesc = dstage + ((mb * 2 * kTcSlabBytes + ks * 2 * SBO) >> 4);
+#pragma unroll
+            for (int j = 0; j < R_CTA; j += 256) {
+              constexpr int kFull = 256;
+              const int ncols = R_CTA - j < kFull ? R_CTA - j : kFull;
+              const uint64_t bdesc =
+                  dstage + ((X_SLABS * kTcSlabBytes + (j / 64) * kTcSlabBytes + ks * 2 * SBO) >> 4);
+              ptx::mma_bf16(tmem_base + static_cast<uint32_t>(mb * R_CTA + j), adesc, bdesc,
                             ptx::idesc_bf16_mn_mn(128, static_cast<uint32_t>(ncols)), acc);
             }
           }
         }
         ptx::mma_commit(&bar_empty[s]);  // frees the stage once these MMAs have read it
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
       ptx::mma_commit(&bar_accum);       // accumulators complete (or: everything issued is done)
       if (!ok) ptx::mbar_wait_bounded(&bar_accum, 0, nullptr, kTcDrainLimit);
     }
   } else {
     // ================= epilogue: TMEM -> registers -> global =================
-    const int q = warp & 3;  // TMEM lane quarter this warp may touch
+    const int q = warp & 3;             // TMEM lane quarter this warp may touch
+    const int half = (warp - 2) >> 2;   // which of the quarter's two warps
     bool ok = kb_count > 0;
-    if (ok && !ptx::mbar_wait_bounded(&bar_accum, 0, abort_flag, kTcWaitLimit)) {
-      if (lane == 0 && *abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 300 + warp);
-      *abort_flag = 1;
-      ok = false;
+    if (ok) {
+      // one polling lane per warp, with back-off: this wait lasts the whole main loop
+      int got = 1;
+      if (lane == 0) {
+        got = ptx::mbar_wait_bounded(&bar_accum, 0, abort_flag, kTcWaitLimit, 128) ? 1 : 0;
+        if (!got) {
+          if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 300 + warp);
+          *abort_flag = 1;
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, got, 0) != 0;
     }
     if (ok && *abort_flag == 0) {
       ptx::fence_tc_after_sync();
       float* out = p.out + static_cast<long long>(z) * p.split_stride;
-      for (int mb = 0; mb < p.MB; ++mb) {
+      const bool scale = p.split_k == 1 && p.rho != nullptr;
+      const long long ld = p.ld_out;
+#pragma unroll 1
+      for (int chunk = half; chunk < MB * (R_CTA / 32); chunk += 2) {
+        const int mb = chunk / (R_CTA / 32);
+        const int j = (chunk % (R_CTA / 32)) * 32;
+        const int row0 = r0 + j;
+        if (row0 >= p.r) continue;      // uniform: padding rows
+        uint32_t v[32];
+        ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
+                               static_cast<uint32_t>(mb * R_CTA + j), v);
+        ptx::tmem_ld_wait();
         const int c = c_tile0 + mb * 128 + q * 32 + lane;
-        for (int j = 0; j < p.r_cta; j += 32) {
-          if (r0 + j >= p.r) break;  // uniform: rest of this tile is padding
-          uint32_t v[32];
-          ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
-                                 static_cast<uint32_t>(mb * p.r_cta + j), v);
-          ptx::tmem_ld_wait();
-          if (c < p.n) {
+        float my_rho = 1.f;
+        if (scale && row0 + lane < p.r) my_rho = __ldg(p.rho + row0 + lane);
+        float* dst = out + static_cast<long long>(row0) * ld + c;
+        const int nvalid = p.r - row0 < 32 ? p.r - row0 : 32;
+        if (nvalid == 32) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int row = r0 + j + i;
-              if (row < p.r) {
-                float val = __uint_as_float(v[i]);
-                if (p.split_k == 1 && p.rho != nullptr) val *= __ldg(p.rho + row);
-                out[static_cast<long long>(row) * p.ld_out + c] = val;
-              }
-            }
+          for (int i = 0; i < 32; ++i) {
+            const float val = __uint_as_float(v[i]) * __shfl_sync(0xffffffffu, my_rho, i);
+            if (c < p.n) dst[i * ld] = val;
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float val = __uint_as_float(v[i]) * __shfl_sync(0xffffffffu, my_rho, i);
+            if (c < p.n && i < nvalid) dst[i * ld] = val;
           }
         }
       }

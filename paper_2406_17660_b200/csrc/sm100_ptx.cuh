@@ -39,16 +39,37 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Non-blocking probe of a phase (returns at once, unlike try_wait which may
+// suspend the thread for an implementation-defined time when the phase is open).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait: gives up after `limit_cycles` SM clocks or as soon as *abort is
 // set by another role of this CTA (abort may be NULL).  Returns false on giving up.
+// sleep_ns == 0 spins on test_wait (single-thread pipeline roles: lowest wake-up
+// latency); sleep_ns > 0 backs off between probes (long waits by several warps).
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity,
-                                                  volatile int* abort, long long limit_cycles) {
-  if (mbar_try_wait(bar, parity)) return true;
+                                                  volatile int* abort, long long limit_cycles,
+                                                  unsigned sleep_ns = 0) {
+  if (mbar_test_wait(bar, parity)) return true;
   const long long start = clock64();
+  unsigned spins = 0;
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (abort != nullptr && *abort != 0) return false;
-    if (clock64() - start > limit_cycles) return false;
+    if (mbar_test_wait(bar, parity)) return true;
+    if (sleep_ns != 0) __nanosleep(sleep_ns);
+    if ((++spins & 63u) == 0u || sleep_ns != 0) {
+      if (abort != nullptr && *abort != 0) return false;
+      if (clock64() - start > limit_cycles) return false;
+    }
   }
 }
 
