@@ -16,7 +16,8 @@ constexpr int kSmCount = 148;
 struct TcPlan {
   int r_pad;      // r_blocks * r_cta: width of the gathered operand
   int r_cta, r_blocks;
-  int MB, n_blocks;
+  int MB, n_blocks;   // n_blocks = gridDim.x (CTAs, an even number when pair)
+  bool pair;          // two CTAs share each MMA (cta_group::2)
   int k_blocks, split_k, stages;
   size_t smem_bytes;
   long long ld_part;        // pitch of a split-K partial, elements
@@ -44,29 +45,43 @@ TcPlan make_plan(int64_t T, int64_t n, int r) {
   double best = 1e300;
   p.MB = 1;
   p.split_k = 1;
+  // GRASS_TC_NO_PAIR (diagnostic) keeps every CTA on its own MMA, for A/B timing
+  const bool can_pair = (p.r_cta % 128) == 0 && getenv("GRASS_TC_NO_PAIR") == nullptr;
+  p.pair = false;
   for (int mb = mb_max; mb >= 1; mb /= 2) {
-    const int n_blocks = static_cast<int>((n + mb * 128 - 1) / (mb * 128));
-    const int64_t tiles = static_cast<int64_t>(n_blocks) * p.r_blocks;
-    const double clk_per_block = static_cast<double>(mb) * p.r_cta < 256.0
-                                     ? 256.0 : static_cast<double>(mb) * p.r_cta;
-    const double fixed = 2000.0 + mb * 128.0 * p.r_cta * 4.0 / 64.0;
-    const int max_s = p.k_blocks < 256 ? p.k_blocks : 256;
-    for (int s = 1; s <= max_s; ++s) {
-      const int64_t ctas = tiles * s;
-      const int64_t waves = (ctas + kSmCount - 1) / kSmCount;
-      const double blocks_per_cta = static_cast<double>((p.k_blocks + s - 1) / s);
-      double cost = waves * (blocks_per_cta * clk_per_block + fixed);
-      if (s > 1) cost += 8.0 * s * static_cast<double>(r) * n / hbm_bytes_per_clk;
-      if (cost < best) {
-        best = cost;
-        p.MB = mb;
-        p.split_k = s;
+    for (int pair = can_pair ? 1 : 0; pair >= 0; --pair) {
+      if (pair && n <= static_cast<int64_t>(mb) * 128) continue;  // nothing for the second CTA
+      const int cta_cols = mb * 128 * (pair ? 2 : 1);
+      const int n_tiles = static_cast<int>((n + cta_cols - 1) / cta_cols);
+      const int64_t tiles = static_cast<int64_t>(n_tiles) * p.r_blocks * (pair ? 2 : 1);  // CTAs
+      // clocks per 32-token block: tensor time, or (single CTA) the shared-memory ceiling
+      double clk_per_block = static_cast<double>(mb) * p.r_cta;
+      if (!pair) clk_per_block *= 1.4;
+      if (clk_per_block < 256.0) clk_per_block = 256.0;
+      const double fixed = 3000.0 + mb * 128.0 * p.r_cta * 4.0 / 128.0;
+      const int max_s = p.k_blocks < 256 ? p.k_blocks : 256;
+      for (int s = 1; s <= max_s; ++s) {
+        const int64_t ctas = tiles * s;
+        const int64_t waves = (ctas + kSmCount - 1) / kSmCount;
+        const double blocks_per_cta = static_cast<double>((p.k_blocks + s - 1) / s);
+        double cost = waves * (blocks_per_cta * clk_per_block + fixed);
+        if (s > 1) cost += 8.0 * s * static_cast<double>(r) * n / hbm_bytes_per_clk;
+        if (cost < best) {
+          best = cost;
+          p.MB = mb;
+          p.split_k = s;
+          p.pair = pair != 0;
+        }
       }
     }
   }
-  p.n_blocks = static_cast<int>((n + p.MB * 128 - 1) / (p.MB * 128));
-  p.stages = tc_stages(p.MB, p.r_cta / 64);
-  p.smem_bytes = static_cast<size_t>(p.stages) * tc_stage_bytes(p.MB, p.r_cta / 64) + 1024;
+  {
+    const int cta_cols = p.MB * 128 * (p.pair ? 2 : 1);
+    p.n_blocks = static_cast<int>((n + cta_cols - 1) / cta_cols) * (p.pair ? 2 : 1);
+  }
+  const int a_slabs = p.pair ? p.r_cta / 128 : p.r_cta / 64;
+  p.stages = tc_stages(p.MB, a_slabs);
+  p.smem_bytes = static_cast<size_t>(p.stages) * tc_stage_bytes(p.MB, a_slabs) + 1024;
   p.ld_part = static_cast<long long>(round_up(static_cast<size_t>(n), 4));
   p.ag_bytes = round_up(static_cast<size_t>(T) * p.r_pad * sizeof(__nv_bfloat16), 256);
   p.part_bytes = p.split_k > 1
@@ -105,36 +120,53 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
   return true;
 }
 
-template <int MB, int NSLAB>
+template <int MB, int NSLAB, bool PAIR>
 int launch_tc_one(dim3 grid, size_t smem, cudaStream_t s, const CUtensorMap& tmX,
                   const CUtensorMap& tmA, const TcParams& p) {
   static bool attr_set[64] = {false};
   int dev = 0;
   GRASS_CUDA_TRY(cudaGetDevice(&dev));
   if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel<MB, NSLAB>,
+    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel<MB, NSLAB, PAIR>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kTcSmemBudget));
     attr_set[dev] = true;
   }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   {
     ProfileScope prof(GRASS_K_PROJECT_TC, s);
-    project_tc_kernel<MB, NSLAB><<<grid, kTcThreads, smem, s>>>(tmX, tmA, p);
+    GRASS_CUDA_TRY(cudaLaunchKernelEx(&cfg, project_tc_kernel<MB, NSLAB, PAIR>, tmX, tmA, p));
   }
-  GRASS_LAUNCH_CHECK();
   return GRASS_OK;
 }
 
-// (MB, NSLAB) with MB * 64 * NSLAB <= 512 TMEM columns.
-int launch_tc(int MB, int nslab, dim3 grid, size_t smem, cudaStream_t s, const CUtensorMap& tmX,
-              const CUtensorMap& tmA, const TcParams& p) {
-#define GRASS_TC_CASE(mb, ns) \
-  if (MB == mb && nslab == ns) return launch_tc_one<mb, ns>(grid, smem, s, tmX, tmA, p)
+// (MB, NSLAB) with MB * 64 * NSLAB <= 512 TMEM columns; pairs need an even NSLAB.
+int launch_tc(int MB, int nslab, bool pair, dim3 grid, size_t smem, cudaStream_t s,
+              const CUtensorMap& tmX, const CUtensorMap& tmA, const TcParams& p) {
+#define GRASS_TC_CASE(mb, ns)                                                                  \
+  if (MB == mb && nslab == ns && !pair)                                                        \
+    return launch_tc_one<mb, ns, false>(grid, smem, s, tmX, tmA, p)
+#define GRASS_TC_PAIR(mb, ns)                                                                  \
+  if (MB == mb && nslab == ns && pair) return launch_tc_one<mb, ns, true>(grid, smem, s, tmX, tmA, p)
   GRASS_TC_CASE(1, 1); GRASS_TC_CASE(1, 2); GRASS_TC_CASE(1, 3); GRASS_TC_CASE(1, 4);
   GRASS_TC_CASE(1, 5); GRASS_TC_CASE(1, 6); GRASS_TC_CASE(1, 7); GRASS_TC_CASE(1, 8);
   GRASS_TC_CASE(2, 1); GRASS_TC_CASE(2, 2); GRASS_TC_CASE(2, 3); GRASS_TC_CASE(2, 4);
   GRASS_TC_CASE(4, 1); GRASS_TC_CASE(4, 2);
+  GRASS_TC_PAIR(1, 2); GRASS_TC_PAIR(1, 4); GRASS_TC_PAIR(1, 6); GRASS_TC_PAIR(1, 8);
+  GRASS_TC_PAIR(2, 2); GRASS_TC_PAIR(2, 4); GRASS_TC_PAIR(4, 2);
 #undef GRASS_TC_CASE
+#undef GRASS_TC_PAIR
   return GRASS_ERR_UNSUPPORTED;
 }
 
@@ -181,8 +213,9 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   p.status = status;
   if (getenv("GRASS_DEBUG_PLAN") != nullptr)
     fprintf(stderr, "grass plan T=%lld n=%lld r=%d: r_cta=%d r_blocks=%d MB=%d n_blocks=%d "
-                    "split_k=%d stages=%d\n", static_cast<long long>(T), static_cast<long long>(n),
-            r, plan.r_cta, plan.r_blocks, plan.MB, plan.n_blocks, plan.split_k, plan.stages);
+                    "split_k=%d stages=%d pair=%d\n", static_cast<long long>(T), static_cast<long long>(n),
+            r, plan.r_cta, plan.r_blocks, plan.MB, plan.n_blocks, plan.split_k, plan.stages,
+            plan.pair ? 1 : 0);
   if (plan.split_k == 1) {
     p.out = Gc;
     p.ld_out = ldgc;
@@ -196,7 +229,7 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   }
   dim3 grid(static_cast<unsigned>(plan.n_blocks), static_cast<unsigned>(plan.r_blocks),
             static_cast<unsigned>(plan.split_k));
-  const int rc = launch_tc(plan.MB, plan.r_cta / 64, grid, plan.smem_bytes, s, tmX, tmA, p);
+  const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, grid, plan.smem_bytes, s, tmX, tmA, p);
   if (rc != GRASS_OK) return rc;
   if (plan.split_k > 1) {
     const int vec = (n % 4 == 0) && (ldgc % 4 == 0) && aligned_to(Gc, 16);

@@ -24,6 +24,15 @@
 // producer and of the MMA issuer bounds the pipeline: tile shape and stage
 // count are template parameters so that every descriptor is a constant plus
 // the stage offset and the loops unroll.
+//
+// PAIR = true runs two CTAs of a cluster as one tcgen05 "CTA pair"
+// (cta_group::2): M = 256 (each CTA holds its own 128 columns of n in its own
+// TMEM), and the B operand is split between the two CTAs, each staging only
+// half of the selected rows.  Shared-memory traffic per SM drops from
+// 96 B/clk of MMA reads + 80 B/clk of TMA writes (above the 128 B/clk an SM
+// can move) to 64 + 48.  The even CTA issues the MMAs for both; both CTAs' TMA
+// loads report to the even CTA's "full" barrier; tcgen05.commit signals the
+// "empty" and "accumulator ready" barriers of both CTAs.  No load is multicast.
 // Every mbarrier wait is bounded; on expiry the CTA records GRASS_ERR_TIMEOUT,
 // drains what it has in flight (bounded again), frees its TMEM and returns.
 #pragma once
@@ -59,17 +68,20 @@ struct TcParams {
   int* status;
 };
 
-template <int MB, int NSLAB>
+template <int MB, int NSLAB, bool PAIR>
 __global__ void __launch_bounds__(kTcThreads, 1)
 project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA,
                   const TcParams p) {
-  constexpr int R_CTA = 64 * NSLAB;
+  constexpr int R_CTA = 64 * NSLAB;          // selected rows per CTA tile (per pair if PAIR)
   constexpr int X_SLABS = 2 * MB;
-  constexpr int N_SLABS = X_SLABS + NSLAB;
-  constexpr int STAGE_BYTES = tc_stage_bytes(MB, NSLAB);
-  constexpr int STAGES = tc_stages(MB, NSLAB);
+  constexpr int A_SLABS = PAIR ? NSLAB / 2 : NSLAB;   // slabs of the gathered operand this CTA stages
+  constexpr int N_SLABS = X_SLABS + A_SLABS;
+  constexpr int STAGE_BYTES = tc_stage_bytes(MB, A_SLABS);
+  constexpr int STAGES = tc_stages(MB, A_SLABS);
+  constexpr int UMMA_M = PAIR ? 256 : 128;
   static_assert(MB * R_CTA <= 512, "accumulators exceed TMEM");
   static_assert(N_SLABS <= 32, "one producer lane per slab");
+  static_assert(!PAIR || NSLAB % 2 == 0, "a CTA pair splits the selected rows in halves of 64k");
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kTcMaxStages];
@@ -81,7 +93,11 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                               ~static_cast<uintptr_t>(1023));
-  const int c_tile0 = blockIdx.x * (MB * 128);
+  // PAIR: CTA `rank` of pair `blockIdx.x / 2` owns, for each of its MB blocks, the 128 columns
+  // pair_base + (mb * 2 + rank) * 128; otherwise the CTA owns MB consecutive blocks.
+  const int rank = PAIR ? static_cast<int>(ptx::cluster_ctarank()) : 0;
+  const int c_base = PAIR ? (blockIdx.x >> 1) * (2 * MB * 128) + rank * 128 : blockIdx.x * (MB * 128);
+  constexpr int C_STEP = PAIR ? 256 : 128;   // columns between this CTA's consecutive blocks
   const int r0 = blockIdx.y * R_CTA;
   // this CTA's token blocks: [kb_begin, kb_begin + kb_count)
   const int kb_per = p.k_blocks / p.split_k, kb_rem = p.k_blocks % p.split_k;
@@ -102,11 +118,16 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     ptx::prefetch_tensormap(&tmA);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(&s_tmem_base, 512);
-    ptx::tmem_relinquish();
+    if (PAIR) {
+      ptx::tmem_alloc_pair(&s_tmem_base, 512);
+      ptx::tmem_relinquish_pair();
+    } else {
+      ptx::tmem_alloc(&s_tmem_base, 512);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::fence_tc_before_sync();
-  __syncthreads();
+  if (PAIR) ptx::cluster_sync_all(); else __syncthreads();
   ptx::fence_tc_after_sync();
   const uint32_t tmem_base = s_tmem_base;
   volatile int* abort_flag = &s_abort;
@@ -115,7 +136,17 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     // ================= TMA producer: one lane per slab =================
     const bool is_x = lane < X_SLABS;
     const CUtensorMap* map = is_x ? &tmX : &tmA;
-    const int xcoord = is_x ? c_tile0 + lane * 64 : r0 + (lane - X_SLABS) * 64;
+    int xcoord;
+    if (is_x) {
+      xcoord = c_base + (lane >> 1) * C_STEP + (lane & 1) * 64;
+    } else if (PAIR) {
+      // slab a of this CTA: 256-row chunk a/2 of the tile, this CTA's half of it
+      const int a = lane - X_SLABS, q = a >> 1;
+      const int wq = R_CTA - 256 * q < 256 ? R_CTA - 256 * q : 256;
+      xcoord = r0 + 256 * q + rank * (wq >> 1) + (a & 1) * 64;
+    } else {
+      xcoord = r0 + (lane - X_SLABS) * 64;
+    }
     uint8_t* my_dst = tiles + lane * kTcSlabBytes;
     int tok = kb_begin * kTcBK;
     int s = 0, issued = 0;
@@ -125,7 +156,9 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       if (lane == 0) {
         ok = ptx::mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kTcWaitLimit) ? 1 : 0;
         if (ok) {
-          ptx::mbar_arrive_expect_tx(&bar_full[s], STAGE_BYTES);
+          // PAIR: the even CTA's barrier collects the bytes of both CTAs
+          if (!PAIR) ptx::mbar_arrive_expect_tx(&bar_full[s], STAGE_BYTES);
+          else if (rank == 0) ptx::mbar_arrive_expect_tx(&bar_full[s], 2 * STAGE_BYTES);
         } else {
           if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 100 + s);
           *abort_flag = 1;
@@ -133,12 +166,15 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
-      if (lane < N_SLABS) ptx::tma_load_2d(my_dst + s * STAGE_BYTES, map, xcoord, tok, &bar_full[s]);
+      if (lane < N_SLABS) {
+        if (PAIR) ptx::tma_load_2d_pair(my_dst + s * STAGE_BYTES, map, xcoord, tok, &bar_full[s]);
+        else ptx::tma_load_2d(my_dst + s * STAGE_BYTES, map, xcoord, tok, &bar_full[s]);
+      }
       tok += kTcBK;
       issued = it + 1;
       if (++s == STAGES) { s = 0; ph ^= 1u; }
     }
-    if (lane == 0 && *abort_flag != 0) {
+    if (lane == 0 && *abort_flag != 0 && rank == 0) {
       // let the copies already issued land before the CTA gives its smem back
       const int first = issued > STAGES ? issued - STAGES : 0;
       for (int it = first; it < issued; ++it)
@@ -146,8 +182,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                                nullptr, kTcDrainLimit);
     }
   } else if (warp == 1) {
-    // ================= MMA issuer: one thread =================
-    if (lane == 0) {
+    // ================= MMA issuer: one thread (of the even CTA if PAIR) =================
+    if (lane == 0 && rank == 0) {
       constexpr uint32_t LBO = kTcSlabBytes, SBO = 1024;
       const uint64_t desc0 = ptx::smem_desc_mn_sw128(ptx::smem_u32(tiles), LBO, SBO);
       bool ok = true;
@@ -173,17 +209,23 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             for (int j = 0; j < R_CTA; j += 256) {
               constexpr int kFull = 256;
               const int ncols = R_CTA - j < kFull ? R_CTA - j : kFull;
+              // slabs of this 256-row chunk in a CTA's stage: 4 per chunk, or 2 when split over a pair
+              const int bslab = PAIR ? (j / 256) * 2 : j / 64;
               const uint64_t bdesc =
-                  dstage + ((X_SLABS * kTcSlabBytes + (j / 64) * kTcSlabBytes + ks * 2 * SBO) >> 4);
-              ptx::mma_bf16(tmem_base + static_cast<uint32_t>(mb * R_CTA + j), adesc, bdesc,
-                            ptx::idesc_bf16_mn_mn(128, static_cast<uint32_t>(ncols)), acc);
+                  dstage + ((X_SLABS * kTcSlabBytes + bslab * kTcSlabBytes + ks * 2 * SBO) >> 4);
+              const uint32_t idesc = ptx::idesc_bf16_mn_mn(UMMA_M, static_cast<uint32_t>(ncols));
+              const uint32_t d = tmem_base + static_cast<uint32_t>(mb * R_CTA + j);
+              if (PAIR) ptx::mma_bf16_pair(d, adesc, bdesc, idesc, acc);
+              else ptx::mma_bf16(d, adesc, bdesc, idesc, acc);
             }
           }
         }
-        ptx::mma_commit(&bar_empty[s]);  // frees the stage once these MMAs have read it
+        // frees the stage (in both CTAs if PAIR) once these MMAs have read it
+        if (PAIR) ptx::mma_commit_pair(&bar_empty[s]); else ptx::mma_commit(&bar_empty[s]);
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
-      ptx::mma_commit(&bar_accum);       // accumulators complete (or: everything issued is done)
+      // accumulators complete (or: everything issued is done)
+      if (PAIR) ptx::mma_commit_pair(&bar_accum); else ptx::mma_commit(&bar_accum);
       if (!ok) ptx::mbar_wait_bounded(&bar_accum, 0, nullptr, kTcDrainLimit);
     }
   } else {
@@ -218,7 +260,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                static_cast<uint32_t>(mb * R_CTA + j), v);
         ptx::tmem_ld_wait();
-        const int c = c_tile0 + mb * 128 + q * 32 + lane;
+        const int c = c_base + mb * C_STEP + q * 32 + lane;
         float my_rho = 1.f;
         if (scale && row0 + lane < p.r) my_rho = __ldg(p.rho + row0 + lane);
         float* dst = out + static_cast<long long>(row0) * ld + c;
@@ -239,11 +281,14 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       }
     }
   }
+  __syncwarp();
   ptx::fence_tc_before_sync();
-  __syncthreads();
+  // PAIR: neither CTA may leave (or free TMEM) while the other can still read its shared
+  // memory through the MMA or signal its barriers
+  if (PAIR) ptx::cluster_sync_all(); else __syncthreads();
   if (warp == 1) {
     ptx::fence_tc_after_sync();
-    ptx::tmem_dealloc(tmem_base, 512);
+    if (PAIR) ptx::tmem_dealloc_pair(tmem_base, 512); else ptx::tmem_dealloc(tmem_base, 512);
   }
 }
 
