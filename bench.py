@@ -251,19 +251,33 @@ def run_gpu(args):
         dY = syn.make_dY(wl.T, m, wl.dtype, proj=pi, device=dev, ld=syn.pad_to(m, 8))
         X = syn.make_X(wl.T, n, wl.dtype, proj=pi, device=dev, ld=syn.pad_to(n, 8))
         block_in.append((dY, X))
-    ws = GrassWorkspace([(m, n) for _, m, n in wl.shapes], wl.T, wl.r, wl.dtype, wl.method, device=dev)
+    # Layers are independent, so consecutive layers go to alternating streams (each with its own
+    # scratch): the HBM-bound kernels of one layer (column gather, Adam, apply) then run beside
+    # the tensor-bound GEMM of its neighbour.  --streams 1 puts everything on one stream.
+    n_streams = max(1, args.streams)
+    main_stream = torch.cuda.current_stream()
+    streams = [main_stream] + [torch.cuda.Stream() for _ in range(n_streams - 1)]
+    wss = [GrassWorkspace([(m, n) for _, m, n in wl.shapes], wl.T, wl.r, wl.dtype, wl.method,
+                          device=dev) for _ in range(n_streams)]
     layers = []
-    for li, pi, name, m, n in wl.layer_list():
+    for i, (li, pi, name, m, n) in enumerate(wl.layer_list()):
         W = syn.make_W(m, n, wl.dtype, layer=li, proj=pi, device=dev, ld=syn.pad_to(n, 8))
-        layers.append((pi, GrassLayer(W, min(wl.r, m), wl.method, K, wl.alpha, wl.lr, wl.beta1,
-                                      wl.beta2, wl.eps, reset_state=wl.reset_state, seed=0,
-                                      layer_id=li * len(wl.shapes) + pi, workspace=ws)))
+        layer = GrassLayer(W, min(wl.r, m), wl.method, K, wl.alpha, wl.lr, wl.beta1, wl.beta2,
+                           wl.eps, reset_state=wl.reset_state, seed=0,
+                           layer_id=li * len(wl.shapes) + pi, workspace=wss[i % n_streams])
+        layer.stream = streams[i % n_streams]
+        layers.append((pi, layer))
     in_bytes = sum(d.numel() * d.element_size() + x.numel() * x.element_size() for d, x in block_in)
 
     def one_step():
+        for st in streams[1:]:
+            st.wait_stream(main_stream)
         for pi, layer in layers:
             dY, X = block_in[pi]
-            layer.step(dY, X)
+            with torch.cuda.stream(layer.stream):
+                layer.step(dY, X)
+        for st in streams[1:]:
+            main_stream.wait_stream(st)
 
     def rewind():
         for _, layer in layers:
@@ -299,10 +313,17 @@ def run_gpu(args):
     rewind()
     n_refresh = (args.steps + K - 1) // K
     cap = args.steps * len(layers) * 5 + n_refresh * len(layers) * 8 + 16
+    # one stream for this pass: an event pair must bracket one kernel running alone, not a kernel
+    # sharing the GPU with another layer's kernels
+    saved_streams = [layer.stream for _, layer in layers]
+    for _, layer in layers:
+        layer.stream = main_stream
     grass.grass_profile_begin(cap)
     for i in range(args.steps):
         one_step()
     launches, recs = grass.grass_profile_end()
+    for (_, layer), st in zip(layers, saved_streams):
+        layer.stream = st
     clocks = sampler.stop() if rank == 0 else None
     per_kernel = {}
     for name, ms in recs:
@@ -365,28 +386,37 @@ def run_gpu(args):
             host_in.append((hd, hx))
         stage = [(torch.empty_like(d), torch.empty_like(x)) for d, x in block_in]
         max_rn = max(l.Gc.numel() for _, l in layers)
-        host_out = torch.empty(max_rn, dtype=torch.float32, pin_memory=True)
+        host_out = [torch.empty(max_rn, dtype=torch.float32, pin_memory=True) for _ in wl.shapes]
         e2e_steps = min(args.steps, args.e2e_steps)
         h2d = sum(d.numel() * d.element_size() + x.numel() * x.element_size()
                   for d, x in host_in) * wl.layers
         d2h = sum(l.Gc.numel() * 4 for _, l in layers)
 
         def e2e_step():
+            for st in streams[1:]:
+                st.wait_stream(main_stream)
             for pi, layer in layers:
                 sd, sx = stage[pi]
-                sd.copy_(host_in[pi][0], non_blocking=True)
-                sx.copy_(host_in[pi][1], non_blocking=True)
-                layer.step(sd, sx)
-                host_out[: layer.Gc.numel()].copy_(layer.Gc.view(-1), non_blocking=True)
+                with torch.cuda.stream(layer.stream):
+                    sd.copy_(host_in[pi][0], non_blocking=True)
+                    sx.copy_(host_in[pi][1], non_blocking=True)
+                    layer.step(sd, sx)
+                    host_out[pi][: layer.Gc.numel()].copy_(layer.Gc.view(-1), non_blocking=True)
+
+        def e2e_join():
+            for st in streams[1:]:
+                main_stream.wait_stream(st)
 
         rewind()
         e2e_step()
+        e2e_join()
         rewind()
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(e2e_steps):
             e2e_step()
+            e2e_join()
         e1.record()
         barrier()
         e2e_ms = aggregate_max(e0.elapsed_time(e1), dist if world > 1 else None)
@@ -423,6 +453,7 @@ def run_gpu(args):
                        "inputs": "one block of distinct dY/X reused by every block",
                        "l2": f"inputs {in_bytes / 1e6:.0f} MB per step, larger than the 126 MB L2",
                        "parallelism": "replicas" if world > 1 else "single GPU",
+                       "streams": n_streams,
                        "flops": "2rTn per layer-step + 2mTn per refresh"},
             "us_per_layer_step_regular": None if reg_ms is None else 1e3 * reg_ms / n_layers,
             "us_per_layer_step_refresh": None if ref_ms is None else 1e3 * ref_ms / n_layers,
@@ -448,6 +479,7 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="override the number of blocks")
     ap.add_argument("--refresh-every", type=int, default=None, help="override K")
     ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--streams", type=int, default=2, help="streams that layers alternate over")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

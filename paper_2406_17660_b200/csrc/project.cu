@@ -189,13 +189,15 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   if (!make_map(&tmX, X, T, n, ldx)) return GRASS_ERR_CUDA;
   if (gather) {
     __nv_bfloat16* Ag = reinterpret_cast<__nv_bfloat16*>(wsp);
-    dim3 ggrid(static_cast<unsigned>((plan.r_pad / 8 + kGatherThreads - 1) / kGatherThreads),
-               static_cast<unsigned>((T + kGatherTokens - 1) / kGatherTokens));
+    const __nv_bfloat16* dYb = static_cast<const __nv_bfloat16*>(dY);
     {
       ProfileScope prof(GRASS_K_GATHER, s);
-      gather_cols_kernel<<<ggrid, kGatherThreads, 0, s>>>(
-          static_cast<const __nv_bfloat16*>(dY), lddy, static_cast<int>(T), static_cast<int>(m),
-          idx, r, plan.r_pad, Ag, status);
+      const int ni = plan.r_pad >= 256 ? 8 : plan.r_pad / 32;   // r_pad is a multiple of 64
+      dim3 ggrid(static_cast<unsigned>((plan.r_pad + 32 * ni - 1) / (32 * ni)),
+                 static_cast<unsigned>((T + kGatherTokens - 1) / kGatherTokens));
+      gather_cols_kernel<<<ggrid, kGatherThreads, 0, s>>>(dYb, lddy, static_cast<int>(T),
+                                                          static_cast<int>(m), idx, r, plan.r_pad,
+                                                          ni, Ag, status);
     }
     GRASS_LAUNCH_CHECK();
     if (!make_map(&tmA, Ag, T, plan.r_pad, plan.r_pad)) return GRASS_ERR_CUDA;

@@ -293,23 +293,28 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 }
 
 // Ag[t, j] = dY[t, idx[j]] (bf16 bits copied unchanged), zero for r <= j < r_pad.
-// One thread carries 8 consecutive j for a run of tokens: gathered 2-byte loads
-// from one dY row (ascending idx keeps them in few sectors), one 16-byte store.
+// HBM moves 32-byte sectors (16 bf16), so the copy reads 2 T m (1 - (1 - r/m)^16)
+// bytes of dY however it is written; what the kernel controls is how many
+// sector look-ups the load unit performs per useful byte.
 constexpr int kGatherThreads = 256;
-constexpr int kGatherTokens = 32;
+constexpr int kGatherTokens = 32;            // tokens per block
 
+// A warp owns one token at a time and 32 * ni consecutive j: lane l loads
+// j = jb + 32 i + l for i < ni, so one load instruction covers 32 neighbouring
+// selected columns (ascending idx: as few 32-byte sectors as the selection
+// allows) and one store instruction writes 64 contiguous bytes of Ag.
 __global__ void __launch_bounds__(kGatherThreads)
 gather_cols_kernel(const __nv_bfloat16* __restrict__ dY, long long lddy, int T, int m,
-                   const int32_t* __restrict__ idx, int r, int r_pad,
-                   __nv_bfloat16* __restrict__ Ag, int* status) {
-  const int jg = blockIdx.x * kGatherThreads + threadIdx.x;  // group of 8 selected rows
-  if (jg * 8 >= r_pad) return;
+                     const int32_t* __restrict__ idx, int r, int r_pad, int ni,
+                     __nv_bfloat16* __restrict__ Ag, int* status) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int jb = blockIdx.x * (32 * ni);
   int rows[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    const int j = jg * 8 + i;
+    const int j = jb + 32 * i + lane;
     int row = -1;
-    if (j < r) {
+    if (i < ni && j < r) {
       row = __ldg(idx + j);
       if (row < 0 || row >= m) {
         record_status(status, GRASS_ERR_INVALID_ARG, row);
@@ -319,20 +324,19 @@ gather_cols_kernel(const __nv_bfloat16* __restrict__ dY, long long lddy, int T, 
     rows[i] = row;
   }
   const unsigned short* src = reinterpret_cast<const unsigned short*>(dY);
+  unsigned short* dst = reinterpret_cast<unsigned short*>(Ag);
   const int t_begin = blockIdx.y * kGatherTokens;
   const int t_end = t_begin + kGatherTokens < T ? t_begin + kGatherTokens : T;
-#pragma unroll 4
-  for (int t = t_begin; t < t_end; ++t) {
+#pragma unroll 2
+  for (int t = t_begin + warp; t < t_end; t += kGatherThreads / 32) {
     const unsigned short* line = src + static_cast<long long>(t) * lddy;
     unsigned short v[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = rows[i] >= 0 ? __ldg(line + rows[i]) : 0;
-    uint4 pack;
-    pack.x = v[0] | (static_cast<uint32_t>(v[1]) << 16);
-    pack.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
-    pack.z = v[4] | (static_cast<uint32_t>(v[5]) << 16);
-    pack.w = v[6] | (static_cast<uint32_t>(v[7]) << 16);
-    *reinterpret_cast<uint4*>(Ag + static_cast<long long>(t) * r_pad + jg * 8) = pack;
+    unsigned short* out = dst + static_cast<long long>(t) * r_pad + jb + lane;
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (i < ni && jb + 32 * i + lane < r_pad) out[32 * i] = v[i];
   }
 }
 

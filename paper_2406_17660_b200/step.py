@@ -54,6 +54,7 @@ class GrassLayer:
         self.U = torch.empty((r, self.n), dtype=torch.float32, device=dev)
         self.Gc = torch.empty((r, self.n), dtype=torch.float32, device=dev)
         self.ws = workspace
+        self.stream = None    # optional: the caller may pin a layer to a stream
         self.t = 0            # iteration counter of Algorithm 1
         self.adam_step = 0    # updates since the state was last zeroed
 
