@@ -1,8 +1,8 @@
 // grass_row_norms: lambda_k = ||G[k,:]||_2 (Section 3.2 of the GRASS paper).
 //
 // HBM-bound streaming reduction: 4 m n bytes in (fp32 G), 4 m out.  A row is
-// owned by TPR threads (32 = one warp for short rows, 256 = one CTA for long
-// ones); each thread issues independent 128-bit loads (four in flight per
+// owned by TPR threads (32 = one warp for short rows ... 256 = one CTA for long
+// ones, chosen so that a thread has at least 16 vector loads to issue); each thread issues independent 128-bit loads (eight in flight per
 // loop trip) into separate fp32 accumulators, then a shuffle tree (and, for a
 // CTA-wide row, one shared-memory hop) finishes the sum.
 #include "common.cuh"
@@ -51,6 +51,15 @@ row_norms_kernel(const T* __restrict__ G, int64_t m, int64_t n, int64_t ldg,
       const V* gv = reinterpret_cast<const V*>(g);
       const int64_t nv = n / N;
       int64_t i = lane_in_row;
+      for (; i + 7 * TPR < nv; i += 8 * TPR) {
+        V v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = __ldg(gv + i + u * TPR);
+        acc0 += Vec<T>::sumsq(v[0]) + Vec<T>::sumsq(v[4]);
+        acc1 += Vec<T>::sumsq(v[1]) + Vec<T>::sumsq(v[5]);
+        acc2 += Vec<T>::sumsq(v[2]) + Vec<T>::sumsq(v[6]);
+        acc3 += Vec<T>::sumsq(v[3]) + Vec<T>::sumsq(v[7]);
+      }
       for (; i + 3 * TPR < nv; i += 4 * TPR) {
         V a = __ldg(gv + i), b = __ldg(gv + i + TPR), c = __ldg(gv + i + 2 * TPR),
           d = __ldg(gv + i + 3 * TPR);
@@ -78,10 +87,11 @@ row_norms_kernel(const T* __restrict__ G, int64_t m, int64_t n, int64_t ldg,
     __shared__ float part[kThreads / 32];
     if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
     __syncthreads();
-    if (threadIdx.x < 32) {
-      float v = threadIdx.x < kThreads / 32 ? part[threadIdx.x] : 0.f;
-      v = warp_sum(v);
-      if (threadIdx.x == 0 && row < m) norms[row] = sqrtf(v);
+    if (lane_in_row == 0 && row < m) {
+      float v = 0.f;
+#pragma unroll
+      for (int w = 0; w < TPR / 32; ++w) v += part[(threadIdx.x >> 5) + w];
+      norms[row] = sqrtf(v);
     }
   }
 }
@@ -90,17 +100,18 @@ template <typename T>
 int launch(const void* G, int64_t m, int64_t n, int64_t ldg, float* norms, cudaStream_t s) {
   const T* g = static_cast<const T*>(G);
   const bool vec = aligned_to(G, 16) && (ldg % Vec<T>::N) == 0;
-  const bool wide = n > 2048;  // long rows: one CTA per row
+  // threads per row: enough 128-bit loads per thread (>= 16) to keep eight in flight
+  const int64_t nv = n / Vec<T>::N;
+  const int tpr = nv >= 16 * 256 ? 256 : nv >= 16 * 128 ? 128 : nv >= 16 * 64 ? 64 : 32;
+  const unsigned grid = static_cast<unsigned>((m + kThreads / tpr - 1) / (kThreads / tpr));
   ProfileScope prof(GRASS_K_ROW_NORMS, s);
-  if (wide) {
-    const unsigned grid = static_cast<unsigned>(m);
-    if (vec) row_norms_kernel<T, kThreads, true><<<grid, kThreads, 0, s>>>(g, m, n, ldg, norms);
-    else     row_norms_kernel<T, kThreads, false><<<grid, kThreads, 0, s>>>(g, m, n, ldg, norms);
-  } else {
-    const unsigned grid = static_cast<unsigned>((m + kThreads / 32 - 1) / (kThreads / 32));
-    if (vec) row_norms_kernel<T, 32, true><<<grid, kThreads, 0, s>>>(g, m, n, ldg, norms);
-    else     row_norms_kernel<T, 32, false><<<grid, kThreads, 0, s>>>(g, m, n, ldg, norms);
+#define GRASS_NORMS_CASE(TPR)                                                                   \
+  if (tpr == TPR) {                                                                             \
+    if (vec) row_norms_kernel<T, TPR, true><<<grid, kThreads, 0, s>>>(g, m, n, ldg, norms);     \
+    else     row_norms_kernel<T, TPR, false><<<grid, kThreads, 0, s>>>(g, m, n, ldg, norms);    \
   }
+  GRASS_NORMS_CASE(32) GRASS_NORMS_CASE(64) GRASS_NORMS_CASE(128) GRASS_NORMS_CASE(256)
+#undef GRASS_NORMS_CASE
   GRASS_LAUNCH_CHECK();
   return GRASS_OK;
 }

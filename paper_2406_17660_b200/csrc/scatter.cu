@@ -16,8 +16,7 @@ template <typename T> struct WTraits;
 template <> struct WTraits<float> {
   static constexpr int N = 4;
   using vec = float4;
-  static __device__ __forceinline__ void add_store(float* w, const float* acc) {
-    float4 v = *reinterpret_cast<float4*>(w);
+  static __device__ __forceinline__ void add_store(float* w, float4 v, const float* acc) {
     v.x += acc[0]; v.y += acc[1]; v.z += acc[2]; v.w += acc[3];
     *reinterpret_cast<float4*>(w) = v;
   }
@@ -26,8 +25,7 @@ template <> struct WTraits<float> {
 template <> struct WTraits<__nv_bfloat16> {
   static constexpr int N = 8;
   using vec = uint4;
-  static __device__ __forceinline__ void add_store(__nv_bfloat16* w, const float* acc) {
-    uint4 raw = *reinterpret_cast<uint4*>(w);
+  static __device__ __forceinline__ void add_store(__nv_bfloat16* w, uint4 raw, const float* acc) {
     __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -58,24 +56,37 @@ scatter_kernel(T* __restrict__ W, int64_t m, int64_t n, int64_t ldw, const float
   constexpr int N = WTraits<T>::N;
   T* w = W + static_cast<int64_t>(row) * ldw;
   if (VEC) {
-    const int64_t c = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) * N;
-    if (c >= n) return;
-    float acc[N];
+    // two column chunks per thread, all loads of both issued before any arithmetic
+    const int64_t ca = (static_cast<int64_t>(blockIdx.x) * 2 * kThreads + threadIdx.x) * N;
+    const int64_t cb = ca + static_cast<int64_t>(kThreads) * N;
+    if (ca >= n) return;
+    const bool two = cb < n;
+    float acc[2][N];
 #pragma unroll
-    for (int i = 0; i < N; ++i) acc[i] = 0.f;
+    for (int i = 0; i < N; ++i) acc[0][i] = acc[1][i] = 0.f;
+    typename WTraits<T>::vec wa = *reinterpret_cast<const typename WTraits<T>::vec*>(w + ca), wb;
+    if (two) wb = *reinterpret_cast<const typename WTraits<T>::vec*>(w + cb);
     for (int j = j0; j < r && idx[j] == row; ++j) {
       const float s = alpha * (rho != nullptr ? rho[j] : 1.f);
-      const float4* u = reinterpret_cast<const float4*>(U + static_cast<int64_t>(j) * ldu + c);
+      const float* urow = U + static_cast<int64_t>(j) * ldu;
+      float4 va[N / 4], vb[N / 4];
 #pragma unroll
       for (int q = 0; q < N / 4; ++q) {
-        const float4 v = __ldg(u + q);
-        acc[4 * q + 0] += s * v.x;
-        acc[4 * q + 1] += s * v.y;
-        acc[4 * q + 2] += s * v.z;
-        acc[4 * q + 3] += s * v.w;
+        va[q] = __ldg(reinterpret_cast<const float4*>(urow + ca) + q);
+        if (two) vb[q] = __ldg(reinterpret_cast<const float4*>(urow + cb) + q);
+      }
+#pragma unroll
+      for (int q = 0; q < N / 4; ++q) {
+        acc[0][4 * q + 0] += s * va[q].x; acc[0][4 * q + 1] += s * va[q].y;
+        acc[0][4 * q + 2] += s * va[q].z; acc[0][4 * q + 3] += s * va[q].w;
+        if (two) {
+          acc[1][4 * q + 0] += s * vb[q].x; acc[1][4 * q + 1] += s * vb[q].y;
+          acc[1][4 * q + 2] += s * vb[q].z; acc[1][4 * q + 3] += s * vb[q].w;
+        }
       }
     }
-    WTraits<T>::add_store(w + c, acc);
+    WTraits<T>::add_store(w + ca, wa, acc[0]);
+    if (two) WTraits<T>::add_store(w + cb, wb, acc[1]);
   } else {
     const int64_t c0 = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) * N;
     for (int64_t c = c0; c < c0 + N && c < n; ++c) {
@@ -96,8 +107,9 @@ int launch(void* W, int64_t m, int64_t n, int64_t ldw, const float* U, int64_t l
   if (status == nullptr) GRASS_CUDA_TRY(err);
   const bool vec = (n % N == 0) && (ldw % N == 0) && (ldu % 4 == 0) && aligned_to(W, 16) &&
                    aligned_to(U, 16);
-  dim3 grid(static_cast<unsigned>((n + kThreads * N - 1) / (kThreads * N)),
-            static_cast<unsigned>(r));
+  // vector path: a thread covers two chunks of N columns; scalar path: one
+  const int64_t per_block = static_cast<int64_t>(kThreads) * N * (vec ? 2 : 1);
+  dim3 grid(static_cast<unsigned>((n + per_block - 1) / per_block), static_cast<unsigned>(r));
   ProfileScope prof(GRASS_K_SCATTER, s);
   if (vec)
     scatter_kernel<T, true><<<grid, kThreads, 0, s>>>(static_cast<T*>(W), m, n, ldw, U, ldu, idx,
