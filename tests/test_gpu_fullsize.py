@@ -1,0 +1,74 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The fp64 oracle cannot form the whole r x n result at T = 32768..65536 in seconds, so whole output
+rows are sampled: for a selected row j the oracle's G_C[j, :] = rho_j * X^T dY[:, sigma_j] is one
+matrix-vector product, Adam and the apply step are row-local, and the row's new W follows.  The
+tensor-core kernel's tiles, CTA pairs and split-K slices all contribute to every sampled row.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2406_17660_b200 as grass
+from paper_2406_17660_b200 import synthetic as syn
+from oracle import grass_oracle as oracle
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def f64(t):
+    return t.detach().to("cpu", torch.float32).numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("T,m,n,r,method", [
+    (32768, 4096, 4096, 1024, grass.SEL_TOPR),              # 7B q: CTA pairs, 2 row blocks, split-K 2
+    (32768, 4096, 11008, 1024, grass.SEL_TOPR),             # 7B down: 86 n-tiles, split-K 4
+    (65536, 1376, 512, 128, grass.SEL_MULTINOMIAL_NORM),    # 60M gate: 4 n-blocks per CTA, 64 splits
+])
+def test_layer_step_on_sampled_rows(T, m, n, r, method):
+    dt = torch.bfloat16
+    X = syn.make_X(T, n, dt, seed0=11)
+    dY = syn.make_dY(T, m, dt, seed0=11)
+    W = syn.make_W(m, n, dt, seed0=11)
+    Xd, dYd = X.to(DEV), dY.to(DEV)
+    ws = grass.step.GrassWorkspace([(m, n)], T, r, dt, method)
+    layer = grass.GrassLayer(W.to(DEV).clone(), r, method, K=200, alpha=0.25, lr=1e-3,
+                             reset_state=True, seed=5, layer_id=2, workspace=ws)
+    layer.step(dYd, Xd)
+    grass.grass_device_status()
+
+    idx = layer.idx.cpu().numpy()
+    rho = layer.rho.cpu().numpy().astype(np.float64)
+    norms = f64(ws.norms[:m])
+    # the selection, from the GPU's own fp32 norms (same bits on both sides)
+    sigma, rho_ref = oracle.select(norms.astype(np.float32), r, method, seed=5, layer_id=2, epoch=0)
+    assert np.array_equal(idx, sigma)
+    np.testing.assert_allclose(rho, rho_ref, rtol=1e-6)
+    # the norms themselves, on sampled rows of the dense gradient
+    X64 = f64(X)
+    rng = np.random.default_rng(T + n)
+    for k in rng.choice(m, 4, replace=False):
+        g_row = X64.T @ f64(dY[:, k])
+        assert abs(norms[k] - np.linalg.norm(g_row)) <= 1e-4 * np.linalg.norm(g_row)
+    # projected gradient, Adam and the apply step on sampled selected rows
+    W64 = f64(W)
+    Gc, M, V, U, Wn = (f64(t) for t in (layer.Gc, layer.M, layer.V, layer.U, layer.W))
+    picks = rng.choice(r, 6, replace=False)
+    for j in picks:
+        g = rho[j] * (X64.T @ f64(dY[:, idx[j]]))
+        err = np.linalg.norm(Gc[j] - g) / np.linalg.norm(g)
+        assert err <= 1e-2 and err <= 1e-4, err
+        M1, V1, U1 = oracle.adam_update(np.zeros(n), np.zeros(n), g, 1e-3, 0.9, 0.999, 1e-8, 1)
+        assert np.linalg.norm(M[j] - M1) <= 1e-4 * np.linalg.norm(M1)
+        assert np.linalg.norm(V[j] - V1) <= 2e-4 * np.linalg.norm(V1)
+        assert np.linalg.norm(U[j] - U1) <= 1e-3 * np.linalg.norm(U1)
+    for k in np.unique(idx[picks]):
+        js = np.nonzero(idx == k)[0]                     # every repeat of this row
+        upd = sum(0.25 * rho[j] * U[j] for j in js)      # the GPU's own U: isolates the apply step
+        want = oracle.round_to_bf16(W64[k] + upd)
+        ulp = np.ldexp(1.0, np.floor(np.log2(np.maximum(np.abs(want), 2.0 ** -126))).astype(int) - 7)
+        assert np.all(np.abs(Wn[k] - want) <= ulp * 1.0001)
+        assert np.mean(Wn[k] != want) < 0.01
+    untouched = np.setdiff1d(np.arange(m), idx)
+    assert torch.equal(layer.W[untouched].cpu(), W[untouched])
