@@ -184,6 +184,10 @@ def test_project_fp32(T, m, n, r):
     (777, 320, 200, 320, None, {"identity": True}),      # dense gradient, idx = NULL
     (64, 128, 128, 1, None, {}),                         # r = 1
     (31, 64, 64, 64, None, {"with_rho": False}),         # fewer tokens than one block
+    (200, 50, 70, 20, 72, {}),                           # n not a multiple of 8 (padded pitch), odd m
+    (64, 13824, 256, 13824, None, {"identity": True}),   # largest LLaMA row count, dense: 27 row blocks
+    (96, 640, 128, 384, None, {}),                       # 384 rows: MMA chunks of 256 + 128, single CTA
+    (96, 640, 512, 384, None, {}),                       # same through a CTA pair
 ])
 def test_project_bf16_tensor_core(T, m, n, r, ldx, kw):
     got, want = _project_case(T, m, n, r, torch.bfloat16, seed=T + n + r, ldx=ldx, **kw)
