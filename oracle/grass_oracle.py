@@ -28,15 +28,23 @@ brute-force subset search for top-r, Monte-Carlo unbiasedness and the
 closed-form variance for the sampler, torch.optim.Adam for the dense special
 case, the Algorithm-4 form of the loop, the index-coverage value printed in
 the paper's appendix and published Philox known-answer vectors.
-Parity unpinned: the Philox counter layout and the ascending output order are
-conventions of this build; nothing in the paper can confirm or refute them.
+Parity unpinned: the Philox counter layout, the ascending output order and the
+exponential-race realisation of the without-replacement variants are
+conventions of this build; nothing in the paper can confirm or refute them
+(the distribution the race produces is pinned against the sequential
+definition).
 """
 from __future__ import annotations
 
 import numpy as np
 
 TOPR = 0
-MULTINOMIAL_NORM = 1
+MULTINOMIAL_NORM = 1       # q ~ lambda,   with replacement, rho = 1/sqrt(r q)
+MULTINOMIAL_NORM2 = 2      # q ~ lambda^2, with replacement, rho = 1/sqrt(r q)
+UNIFORM = 3                # q = 1/m,      with replacement, rho = sqrt(m/r)
+MULTINOMIAL_NORM_NR = 4    # the three distributions without replacement, rho = 1
+MULTINOMIAL_NORM2_NR = 5
+UNIFORM_NR = 6
 
 # Tag placed in the fourth counter word of every Philox call made by select.
 PHILOX_STREAM_TAG = 0x47524153
@@ -132,23 +140,34 @@ def select_topr(norms, r):
     return sigma, rho
 
 
-def select_multinomial_norm(norms, r, seed, layer_id, epoch):
-    """Multinomial-Norm with replacement (Section 3.2 A, Theorem 1).
+def sampling_weights(lam, method):
+    """Unnormalised q of the three sampling distributions of Section 3.2 A."""
+    if method in (MULTINOMIAL_NORM, MULTINOMIAL_NORM_NR):
+        return lam.copy()                       # Multinomial-Norm (Theorem 1)
+    if method in (MULTINOMIAL_NORM2, MULTINOMIAL_NORM2_NR):
+        return lam * lam                        # Multinomial-Norm^2 (subspace preservation)
+    if method in (UNIFORM, UNIFORM_NR):
+        return np.ones_like(lam)                # Uniform
+    raise ValueError("not a sampling method")
 
-    q_k = lambda_k / sum_i lambda_i;  sigma_j i.i.d. ~ Multinomial(1, q);
-    rho_j = 1 / sqrt(r * q_{sigma_j}).  Draw j inverts the running sum
-    c_k = sum_{i<=k} lambda_i at u_j * S with u_j = word_j * 2^-32:
-    sigma_j = min{k : c_k > u_j S}, so a zero-norm row is never drawn.
-    The r pairs are reported ascending by row (repeats kept).
+
+def select_with_replacement(norms, r, method, seed, layer_id, epoch):
+    """Sampling with replacement (Section 3.2 A): sigma_j i.i.d. ~ Multinomial(1, q) with
+    q = w / sum(w), w from sampling_weights; rho_j = 1 / sqrt(r * q_{sigma_j}).
+
+    Draw j inverts the running sum c_k = sum_{i<=k} w_i at u_j * S with
+    u_j = word_j * 2^-32: sigma_j = min{k : c_k > u_j S}, so a zero-weight row
+    is never drawn.  The r pairs are reported ascending by row (repeats kept).
     """
     lam = _check_norms(norms)
     m = lam.shape[0]
     if not 1 <= r <= m:
         raise ValueError("need 1 <= r <= m")
-    c = np.cumsum(lam)
+    w = sampling_weights(lam, method)
+    c = np.cumsum(w)
     S = c[-1]
     if not S > 0:
-        raise DegenerateNorms("all row norms are zero")
+        raise DegenerateNorms("all sampling weights are zero")
     words = draw_words(r, seed, layer_id, epoch)
     sigma = np.empty(r, dtype=np.int64)
     for j in range(r):
@@ -156,16 +175,56 @@ def select_multinomial_norm(norms, r, seed, layer_id, epoch):
         k = int(np.searchsorted(c, u * S, side="right"))
         sigma[j] = min(k, m - 1)
     sigma.sort()
-    q = lam[sigma] / S
+    q = w[sigma] / S
     rho = 1.0 / np.sqrt(r * q)
     return sigma, rho
+
+
+def select_multinomial_norm(norms, r, seed, layer_id, epoch):
+    """Multinomial-Norm with replacement (Section 3.2 A, Theorem 1): q_k = lambda_k / sum(lambda)."""
+    return select_with_replacement(norms, r, MULTINOMIAL_NORM, seed, layer_id, epoch)
+
+
+def nr_scores(norms, method, seed, layer_id, epoch):
+    """Scores whose r largest entries are a sample without replacement.
+
+    The paper's "-NR" variants (Section 3.2 A) draw r distinct rows, each draw
+    from q restricted to the rows not yet drawn, and set rho = 1; it does not
+    say how the draws are made.  This build uses the exponential-race form of
+    that sequential scheme (Efraimidis & Spirakis 2006): row k gets
+    t_k = -log(u_k) / w_k with u_k uniform on (0, 1); the rows with the r
+    smallest t -- equivalently the r largest scores w_k / (-log u_k) -- are
+    distributed exactly as r successive draws without replacement.
+    u_k = (word_k + 1/2) * 2^-32, word_k = Philox word (k mod 4) of block
+    (k div 4, layer_id, epoch, tag).  The score is rounded to fp32 and the
+    decision is taken on those fp32 values (ties to the lower row).
+    """
+    lam = _check_norms(norms)
+    m = lam.shape[0]
+    w = sampling_weights(lam, method)
+    words = draw_words(m, seed, layer_id, epoch).astype(np.float64)
+    u = (words + 0.5) * 2.0 ** -32
+    return (w / -np.log(u)).astype(np.float32)
+
+
+def select_without_replacement(norms, r, method, seed, layer_id, epoch):
+    """The -NR variants: r distinct rows, rho = 1, ascending by row."""
+    lam = _check_norms(norms)
+    m = lam.shape[0]
+    if not 1 <= r <= m:
+        raise ValueError("need 1 <= r <= m")
+    if np.count_nonzero(sampling_weights(lam, method) > 0) < r:
+        raise DegenerateNorms("fewer than r rows have positive weight")
+    return select_topr(nr_scores(norms, method, seed, layer_id, epoch), r)
 
 
 def select(norms, r, method, seed=0, layer_id=0, epoch=0):
     if method == TOPR:
         return select_topr(norms, r)
-    if method == MULTINOMIAL_NORM:
-        return select_multinomial_norm(norms, r, seed, layer_id, epoch)
+    if method in (MULTINOMIAL_NORM, MULTINOMIAL_NORM2, UNIFORM):
+        return select_with_replacement(norms, r, method, seed, layer_id, epoch)
+    if method in (MULTINOMIAL_NORM_NR, MULTINOMIAL_NORM2_NR, UNIFORM_NR):
+        return select_without_replacement(norms, r, method, seed, layer_id, epoch)
     raise ValueError("unknown selection method")
 
 

@@ -309,3 +309,48 @@ def test_memory_accounting_reproduces_13b_example():
                                       seq=256, batch=1, r=128)
     for name, val in _rows("memory_13b.txt"):
         assert round(got[name], 2) == float(val), name
+
+
+# ---- the other sampling distributions of Section 3.2 A ----
+def test_norm2_and_uniform_with_replacement_frequencies_and_rho():
+    lam = np.array([3.0, 0.5, 1.0, 0.0, 2.0, 0.25])
+    r, epochs = 6, 3000
+    for method, w in ((oracle.MULTINOMIAL_NORM2, lam ** 2), (oracle.UNIFORM, np.ones(6))):
+        q = w / w.sum()
+        counts = np.zeros(6)
+        for e in range(epochs):
+            sigma, rho = oracle.select(lam, r, method, seed=5, layer_id=1, epoch=e)
+            counts += np.bincount(sigma, minlength=6)
+            np.testing.assert_allclose(rho, 1 / np.sqrt(r * q[sigma]), rtol=1e-14)
+        nz = q > 0
+        expected = q[nz] * r * epochs
+        chi2 = np.sum((counts[nz] - expected) ** 2 / expected)
+        assert chi2 < 20.5 if nz.sum() == 6 else chi2 < 18.5      # 99.9 % points, 5 and 4 dof
+        assert np.all(counts[~nz] == 0)
+    sigma, rho = oracle.select(lam, 3, oracle.UNIFORM, seed=1)
+    np.testing.assert_allclose(rho, np.sqrt(6 / 3), rtol=1e-14)
+
+
+def test_without_replacement_matches_sequential_sampling_exactly_in_distribution():
+    """The exponential race must give each unordered pair the probability that two successive
+    draws without replacement give it: w_a/S * w_b/(S - w_a) + w_b/S * w_a/(S - w_b)."""
+    lam = np.array([1.0, 2.0, 3.0, 4.0])
+    for method, w in ((oracle.MULTINOMIAL_NORM_NR, lam), (oracle.MULTINOMIAL_NORM2_NR, lam ** 2),
+                      (oracle.UNIFORM_NR, np.ones(4))):
+        S = w.sum()
+        pairs = list(itertools.combinations(range(4), 2))
+        p = np.array([w[a] / S * w[b] / (S - w[a]) + w[b] / S * w[a] / (S - w[b]) for a, b in pairs])
+        assert abs(p.sum() - 1) < 1e-12
+        epochs = 12000
+        counts = np.zeros(len(pairs))
+        for e in range(epochs):
+            sigma, rho = oracle.select(lam, 2, method, seed=99, layer_id=0, epoch=e)
+            assert len(set(sigma)) == 2 and np.all(rho == 1.0) and sigma[0] < sigma[1]
+            counts[pairs.index(tuple(sigma))] += 1
+        chi2 = np.sum((counts - p * epochs) ** 2 / (p * epochs))
+        assert chi2 < 20.5                                         # 99.9 % point, 5 dof
+    # r = m takes every row; too few positive weights is an error
+    assert list(oracle.select(lam, 4, oracle.MULTINOMIAL_NORM_NR, seed=3)[0]) == [0, 1, 2, 3]
+    with pytest.raises(oracle.DegenerateNorms):
+        oracle.select(np.array([1.0, 0.0, 0.0]), 2, oracle.MULTINOMIAL_NORM_NR, seed=3)
+    assert len(oracle.select(np.array([1.0, 0.0, 0.0]), 2, oracle.UNIFORM_NR, seed=3)[0]) == 2
