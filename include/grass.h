@@ -53,8 +53,13 @@ typedef enum {
 typedef enum { GRASS_F32 = 0, GRASS_BF16 = 1 } grass_dtype_t;
 
 typedef enum {
-  GRASS_SEL_TOPR = 0,            /* Section 3.2 B */
-  GRASS_SEL_MULTINOMIAL_NORM = 1 /* Section 3.2 A, Theorem 1 (with replacement) */
+  GRASS_SEL_TOPR = 0,                 /* Section 3.2 B */
+  GRASS_SEL_MULTINOMIAL_NORM = 1,     /* Section 3.2 A, Theorem 1: q ~ norm, with replacement */
+  GRASS_SEL_MULTINOMIAL_NORM2 = 2,    /* q ~ norm^2 (subspace preservation), with replacement */
+  GRASS_SEL_UNIFORM = 3,              /* q = 1/m, with replacement */
+  GRASS_SEL_MULTINOMIAL_NORM_NR = 4,  /* the three distributions without replacement ("-NR") */
+  GRASS_SEL_MULTINOMIAL_NORM2_NR = 5,
+  GRASS_SEL_UNIFORM_NR = 6
 } grass_sel_t;
 
 /*
@@ -72,13 +77,22 @@ int grass_row_norms(const void* G, int dt, int64_t m, int64_t n, int64_t ldg,
  * compute_P (Section 3.2): choose sigma and rho from the row norms.
  *   GRASS_SEL_TOPR: rho = 1, sigma = the r largest norms; equal norms go to
  *     the lower row index.
- *   GRASS_SEL_MULTINOMIAL_NORM: sigma_j i.i.d. ~ Multinomial(1, q), q_k =
- *     lambda_k / sum(lambda), rho_j = 1 / sqrt(r q_{sigma_j}).  Draw j inverts
- *     the fp64 running sum of the norms at u_j * sum, u_j = w_j * 2^-32, where
+ *   With replacement (GRASS_SEL_MULTINOMIAL_NORM, _NORM2, GRASS_SEL_UNIFORM):
+ *     sigma_j i.i.d. ~ Multinomial(1, q), q_k = w_k / sum(w) with w = lambda,
+ *     lambda^2 or 1, rho_j = 1 / sqrt(r q_{sigma_j}).  Draw j inverts
+ *     the fp64 running sum of the weights at u_j * sum, u_j = w_j * 2^-32, where
  *     w_j is word (j mod 4) of Philox4x32-10 with key (seed low, seed high) and
  *     counter (j div 4, layer_id, epoch, 0x47524153): sigma_j = min{k : c_k >
  *     u_j * sum}.  The result is a pure function of (norms, seed, layer_id,
  *     epoch); no generator state is kept.
+ *   Without replacement (the _NR methods): r distinct rows, rho = 1.  The paper
+ *     does not say how the draws are made; here row k scores w_k / (-log u_k),
+ *     u_k = (word_k + 1/2) * 2^-32 with word_k = Philox word (k mod 4) of counter
+ *     (k div 4, layer_id, epoch, 0x47524153), the score is rounded to fp32, and
+ *     the r largest scores win (equal scores: lower row).  This exponential race
+ *     has exactly the distribution of r successive draws, each from q restricted
+ *     to the rows not yet drawn.  Fewer than r rows of positive weight:
+ *     GRASS_ERR_DEGENERATE.
  *   norms  [m] fp32, read only.     idx [r] int32 and rho [r] fp32, written,
  *   ascending by row (repeated rows are adjacent).
  *   ws     scratch of at least grass_select_workspace_bytes(m, r, method)

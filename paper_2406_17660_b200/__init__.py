@@ -6,7 +6,8 @@ Importing the package does not load the library; the first call does, and
 raises if it has not been built.
 """
 from .binding import (  # noqa: F401
-    GrassError, BF16, F32, SEL_TOPR, SEL_MULTINOMIAL_NORM,
+    GrassError, BF16, F32, SEL_TOPR, SEL_MULTINOMIAL_NORM, SEL_MULTINOMIAL_NORM2, SEL_UNIFORM,
+    SEL_MULTINOMIAL_NORM_NR, SEL_MULTINOMIAL_NORM2_NR, SEL_UNIFORM_NR,
     grass_row_norms, grass_select, grass_select_static, grass_select_workspace_bytes,
     grass_project_grad, grass_project_workspace_bytes,
     grass_subspace_adam, grass_scatter_update, grass_device_status,

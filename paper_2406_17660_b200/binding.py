@@ -13,6 +13,8 @@ import torch
 
 F32, BF16 = 0, 1
 SEL_TOPR, SEL_MULTINOMIAL_NORM = 0, 1
+SEL_MULTINOMIAL_NORM2, SEL_UNIFORM = 2, 3
+SEL_MULTINOMIAL_NORM_NR, SEL_MULTINOMIAL_NORM2_NR, SEL_UNIFORM_NR = 4, 5, 6
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None

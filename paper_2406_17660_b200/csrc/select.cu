@@ -1,5 +1,6 @@
-// grass_select: compute_P of the GRASS paper (Section 3.2) -- Top-r, or
-// Multinomial-Norm sampling with replacement and rho_j = 1/sqrt(r q_sigma_j).
+// grass_select: compute_P of the GRASS paper (Section 3.2) -- Top-r; sampling
+// with replacement from q ~ norm, norm^2 or uniform with rho_j = 1/sqrt(r q_sigma_j);
+// and the same three distributions without replacement with rho = 1.
 //
 // m is at most a few tens of thousands and r at most a few thousand, so this
 // is a latency-bound single-CTA kernel (1024 threads); everything it needs to
@@ -12,7 +13,10 @@
 //   Rows above the threshold are taken; rows equal to it are taken lowest row
 //   first until r are chosen.
 //
-//   Multinomial-Norm: fp64 inclusive running sum of the norms (block scan in
+//   Without replacement: every row gets an exponential-race score (one Philox
+//   word per row), and the Top-r machinery ranks the fp32 scores.
+//
+//   With replacement: fp64 inclusive running sum of the weights (block scan in
 //   row order), then one thread per draw: Philox4x32-10 word -> u -> binary
 //   search for min{k : c_k > u S}; hits are counted per row with integer
 //   atomics (order-independent), and a last scan over the counts writes the
@@ -70,6 +74,18 @@ __device__ __forceinline__ uint32_t norm_key(float v) {
   return v == 0.f ? 0u : __float_as_uint(v);  // folds -0 into +0
 }
 
+__device__ __forceinline__ bool is_nr(int method) {
+  return method == GRASS_SEL_MULTINOMIAL_NORM_NR || method == GRASS_SEL_MULTINOMIAL_NORM2_NR ||
+         method == GRASS_SEL_UNIFORM_NR;
+}
+// Unnormalised q of the three sampling distributions (Section 3.2 A), in fp64.
+__device__ __forceinline__ double sampling_weight(int method, float lambda) {
+  const double l = static_cast<double>(lambda);
+  if (method == GRASS_SEL_MULTINOMIAL_NORM2 || method == GRASS_SEL_MULTINOMIAL_NORM2_NR) return l * l;
+  if (method == GRASS_SEL_UNIFORM || method == GRASS_SEL_UNIFORM_NR) return 1.0;
+  return l;
+}
+
 struct SelectArgs {
   const float* norms;
   int m, r, method;
@@ -108,7 +124,34 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
     return;
   }
 
-  if (a.method == GRASS_SEL_TOPR) {
+  const float* keys = a.norms;   // what the r largest are taken of
+  if (is_nr(a.method)) {
+    // ---- without replacement: exponential race (Efraimidis & Spirakis).  Row k scores
+    // w_k / (-log u_k), u_k = (word_k + 1/2) 2^-32; the r largest scores are distributed as r
+    // successive draws without replacement.  Scores are rounded to fp32 and ranked as such. ----
+    float* scores = reinterpret_cast<float*>(a.cdf);
+    int positive = 0;
+    for (int k = tid; k < m; k += kThreads) {
+      const uint4 blk = philox4x32_10(make_uint4(static_cast<uint32_t>(k >> 2), a.layer_id, a.epoch,
+                                                 kStreamTag),
+                                      make_uint2(a.seed_lo, a.seed_hi));
+      const uint32_t sel = k & 3;
+      const uint32_t word = sel == 0 ? blk.x : sel == 1 ? blk.y : sel == 2 ? blk.z : blk.w;
+      const double u = (static_cast<double>(word) + 0.5) * 0x1p-32;
+      const double w = sampling_weight(a.method, a.norms[k]);
+      scores[k] = static_cast<float>(w / -log(u));
+      positive += w > 0.0;
+    }
+    int total_positive;
+    block_inclusive_scan<int>(positive, s_int, total_positive);
+    if (total_positive < r) {
+      if (tid == 0) record_status(a.status, GRASS_ERR_DEGENERATE, total_positive);
+      return;
+    }
+    __syncthreads();
+    keys = scores;
+  }
+  if (a.method == GRASS_SEL_TOPR || is_nr(a.method)) {
     // ---- radix select of the r-th largest key ----
     if (tid == 0) { s_prefix = 0u; s_need = r; }
     for (int pass = 3; pass >= 0; --pass) {
@@ -118,7 +161,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
       const uint32_t prefix = s_prefix;
       const uint32_t himask = pass == 3 ? 0u : (0xffffffffu << (shift + 8));
       for (int k = tid; k < m; k += kThreads) {
-        const uint32_t key = norm_key(a.norms[k]);
+        const uint32_t key = norm_key(keys[k]);
         if ((key & himask) == prefix) atomicAdd(&s_hist[(key >> shift) & 0xff], 1);
       }
       __syncthreads();
@@ -142,7 +185,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
       uint32_t key = 0u;
       int is_eq = 0, is_gt = 0;
       if (k < m) {
-        key = norm_key(a.norms[k]);
+        key = norm_key(keys[k]);
         is_eq = key == tau;
         is_gt = key > tau;
       }
@@ -161,11 +204,11 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
     return;
   }
 
-  // ---- Multinomial-Norm ----
+  // ---- with replacement: inverse CDF of the sampling weights ----
   double carry = 0.0;
   for (int k0 = 0; k0 < m; k0 += kThreads) {
     const int k = k0 + tid;
-    const double v = k < m ? static_cast<double>(a.norms[k]) : 0.0;
+    const double v = k < m ? sampling_weight(a.method, a.norms[k]) : 0.0;
     double total;
     const double incl = block_inclusive_scan<double>(v, s_dbl, total);
     if (k < m) {
@@ -202,7 +245,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
     int total;
     const int incl = block_inclusive_scan<int>(cnt, s_int, total);
     if (cnt > 0) {
-      const double q = static_cast<double>(a.norms[k]) / S;
+      const double q = sampling_weight(a.method, a.norms[k]) / S;
       const float rho = static_cast<float>(1.0 / sqrt(static_cast<double>(r) * q));
       const int pos = out_base + incl - cnt;
       for (int i = 0; i < cnt; ++i) {
@@ -233,8 +276,7 @@ extern "C" int grass_select(const float* norms, int64_t m, int32_t r, int method
   if (norms == nullptr || idx == nullptr || rho == nullptr || m < 1 || m > 0x7fffffffLL ||
       r < 1 || r > m)
     return GRASS_ERR_INVALID_ARG;
-  if (method != GRASS_SEL_TOPR && method != GRASS_SEL_MULTINOMIAL_NORM)
-    return GRASS_ERR_UNSUPPORTED;
+  if (method < GRASS_SEL_TOPR || method > GRASS_SEL_UNIFORM_NR) return GRASS_ERR_UNSUPPORTED;
   SelectArgs a;
   a.cdf = nullptr;
   a.counts = nullptr;
@@ -311,8 +353,7 @@ extern "C" int grass_select_static(const float* norms, int64_t m, int32_t r, int
             static_cast<long long>(m), kStaticMaxM);
     return GRASS_ERR_WORKSPACE;
   }
-  if (method != GRASS_SEL_TOPR && method != GRASS_SEL_MULTINOMIAL_NORM)
-    return GRASS_ERR_UNSUPPORTED;
+  if (method < GRASS_SEL_TOPR || method > GRASS_SEL_UNIFORM_NR) return GRASS_ERR_UNSUPPORTED;
   unsigned char* scratch = nullptr;
   const int rc = static_scratch(&scratch);
   if (rc != GRASS_OK) return rc;

@@ -124,6 +124,51 @@ def test_select_multinomial_matches_oracle(m, r, seed, layer_id, epoch):
     _check_multinomial(_lognormal_norms(m, m * 3 + r, zeros=m // 8), r, seed, layer_id, epoch)
 
 
+@pytest.mark.parametrize("method", [grass.SEL_MULTINOMIAL_NORM2, grass.SEL_UNIFORM])
+@pytest.mark.parametrize("m,r", [(512, 128), (5461, 512), (13824, 1024)])
+def test_select_other_distributions_with_replacement(method, m, r):
+    lam = _lognormal_norms(m, m + r + method, zeros=m // 8)
+    status, idx, rho = _gpu_select(lam, r, method, seed=21, layer_id=6, epoch=3)
+    assert status == 0
+    sigma, rho_ref = oracle.select(lam, r, method, seed=21, layer_id=6, epoch=3)
+    if not np.array_equal(idx, sigma):
+        w = oracle.sampling_weights(lam.astype(np.float64), method)
+        c = np.cumsum(w)
+        u = oracle.draw_words(r, 21, 6, 3).astype(np.float64) * 2.0 ** -32 * c[-1]
+        gap = np.min(np.abs(c[None, :] - u[:, None]), axis=1) / c[-1]
+        assert np.sum(idx != sigma) <= np.sum(gap < 1e-6)
+    else:
+        np.testing.assert_allclose(rho, rho_ref, rtol=1e-6)
+
+
+@pytest.mark.parametrize("method", [grass.SEL_MULTINOMIAL_NORM_NR, grass.SEL_MULTINOMIAL_NORM2_NR,
+                                    grass.SEL_UNIFORM_NR])
+@pytest.mark.parametrize("m,r", [(512, 128), (2048, 512), (13824, 1024), (300, 260)])
+def test_select_without_replacement(method, m, r):
+    lam = _lognormal_norms(m, m + 5 * r + method, zeros=m // 10)
+    status, idx, rho = _gpu_select(lam, r, method, seed=4242, layer_id=9, epoch=1)
+    assert status == 0
+    sigma, _ = oracle.select(lam, r, method, seed=4242, layer_id=9, epoch=1)
+    assert np.all(rho == 1.0) and len(set(idx.tolist())) == r and np.all(np.diff(idx) > 0)
+    if not np.array_equal(idx, sigma):
+        # allowed only where the fp64 scores at the selection threshold are within 1e-6 relative
+        sc = oracle.nr_scores(lam, method, 4242, 9, 1).astype(np.float64)
+        thr = np.sort(sc)[-r]
+        swapped = np.setxor1d(idx, sigma)
+        assert np.all(np.abs(sc[swapped] - thr) <= 1e-6 * thr), "mismatch beyond the near-tie allowance"
+
+
+def test_select_without_replacement_needs_enough_positive_rows():
+    lam = np.zeros(64, dtype=np.float32)
+    lam[:5] = 1.0
+    status, idx, _ = _gpu_select(lam, 6, grass.SEL_MULTINOMIAL_NORM_NR)
+    assert status == 4 and np.all(idx == -7)
+    status, idx, _ = _gpu_select(lam, 5, grass.SEL_MULTINOMIAL_NORM_NR)
+    assert status == 0 and np.array_equal(idx, np.arange(5))
+    status, idx, _ = _gpu_select(lam, 6, grass.SEL_UNIFORM_NR)
+    assert status == 0
+
+
 def test_select_degenerate_inputs_leave_outputs_untouched():
     lam = _lognormal_norms(100, 1)
     for bad, method in ((np.nan, grass.SEL_TOPR), (np.inf, grass.SEL_TOPR), (-1.0, grass.SEL_TOPR),
