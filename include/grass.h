@@ -163,6 +163,24 @@ int grass_project_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx,
                        void* stream);
 
 /*
+ * Row norms of the weight gradient without forming it (Section 3.1 "Memory
+ * savings" applied to compute_P of Section 3.2):
+ *   norms[k] = || (dY^T X)[k, :] ||_2,   k < m.
+ * The paper's refresh iteration computes the full gradient once to take its row
+ * norms; here the dense GEMM's epilogue reduces the squares of each output tile
+ * and the m x n matrix is never written.  Arguments as for grass_project_grad
+ * with idx = NULL; norms [m] fp32 is written; ws needs
+ * grass_grad_row_norms_workspace_bytes(T, m, n, dt) bytes (GRASS_BF16: m * n / 8
+ * bytes of per-column-group partial sums, added in a fixed order; GRASS_F32: the
+ * fp32 path forms the small gradient in ws and calls grass_row_norms).  The
+ * token sum is not split, so every square is taken of a complete dot product.
+ */
+size_t grass_grad_row_norms_workspace_bytes(int64_t T, int64_t m, int64_t n, int dt);
+int grass_grad_row_norms(const void* dY, int64_t lddy, const void* X, int64_t ldx, int dt,
+                         int64_t T, int64_t m, int64_t n, float* norms, void* ws, size_t ws_bytes,
+                         void* stream);
+
+/*
  * adam.update on the subspace state (Appendix A):
  *   M <- beta1 M + (1 - beta1) Gc;  V <- beta2 V + (1 - beta2) Gc^2;
  *   U = -lr * (M / (1 - beta1^step)) / (sqrt(V / (1 - beta2^step)) + eps).

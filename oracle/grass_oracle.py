@@ -68,6 +68,11 @@ def row_norms(G):
     return np.sqrt(np.sum(G * G, axis=1))
 
 
+def grad_row_norms(dY, X):
+    """Row norms of G_W = dY^T X: what a refresh iteration feeds to compute_P."""
+    return row_norms(dense_grad(dY, X))
+
+
 # --------------------------------------------------------------------------
 # Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as
 # easy as 1, 2, 3", SC'11).  Written out with Python integers.

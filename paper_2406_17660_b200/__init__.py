@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     SEL_MULTINOMIAL_NORM_NR, SEL_MULTINOMIAL_NORM2_NR, SEL_UNIFORM_NR,
     grass_row_norms, grass_select, grass_select_static, grass_select_workspace_bytes,
     grass_project_grad, grass_project_workspace_bytes,
+    grass_grad_row_norms, grass_grad_row_norms_workspace_bytes,
     grass_subspace_adam, grass_scatter_update, grass_device_status,
     grass_status_string, grass_profile_begin, grass_profile_end, library_path, load_library,
 )

@@ -41,6 +41,9 @@ _SIGNATURES = {
     "grass_project_grad": (c_int, [c_void_p, c_int64, c_void_p, c_int64, c_int, c_int64, c_int64,
                                    c_int64, c_void_p, c_void_p, c_int32, c_void_p, c_int64,
                                    c_void_p, c_size_t, c_void_p]),
+    "grass_grad_row_norms_workspace_bytes": (c_size_t, [c_int64, c_int64, c_int64, c_int]),
+    "grass_grad_row_norms": (c_int, [c_void_p, c_int64, c_void_p, c_int64, c_int, c_int64, c_int64,
+                                     c_int64, c_void_p, c_void_p, c_size_t, c_void_p]),
     "grass_subspace_adam": (c_int, [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int64,
                                     c_int32, c_int64, c_double, c_double, c_double, c_double,
                                     c_int32, c_void_p]),
@@ -165,6 +168,22 @@ def grass_project_grad(dY, X, idx, rho, r, Gc, ws) -> None:
     _check(load_library().grass_project_grad(_ptr(dY), _ld(dY), _ptr(X), _ld(X), _dtype_code(X), T,
                                              m, n, _ptr(idx), _ptr(rho), r, _ptr(Gc), _ld(Gc),
                                              _ptr(ws), ws_bytes, _stream()), "grass_project_grad")
+
+
+def grass_grad_row_norms_workspace_bytes(T: int, m: int, n: int, dt: int) -> int:
+    return int(load_library().grass_grad_row_norms_workspace_bytes(T, m, n, dt))
+
+
+def grass_grad_row_norms(dY, X, norms, ws) -> None:
+    T, m = dY.shape
+    T2, n = X.shape
+    if T2 != T or dY.dtype != X.dtype:
+        raise ValueError("dY and X must share the token dimension and dtype")
+    _require(norms, torch.float32, "norms")
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(load_library().grass_grad_row_norms(_ptr(dY), _ld(dY), _ptr(X), _ld(X), _dtype_code(X),
+                                               T, m, n, _ptr(norms), _ptr(ws), ws_bytes, _stream()),
+           "grass_grad_row_norms")
 
 
 def grass_subspace_adam(Gc, M, V, U, lr, beta1, beta2, eps, step) -> None:

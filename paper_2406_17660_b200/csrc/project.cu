@@ -30,7 +30,7 @@ struct TcPlan {
 // n-tiles (MB) make more, smaller CTAs, which cuts partial traffic when the
 // output is tiny; larger ones cut the number of times the gathered operand is
 // re-read.  The result depends only on (T, n, r), so it is reproducible.
-TcPlan make_plan(int64_t T, int64_t n, int r) {
+TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false) {
   TcPlan p;
   const int r64 = static_cast<int>(round_up(static_cast<size_t>(r), 64));
   p.r_blocks = (r64 + 511) / 512;
@@ -59,7 +59,7 @@ TcPlan make_plan(int64_t T, int64_t n, int r) {
       if (!pair) clk_per_block *= 1.4;
       if (clk_per_block < 256.0) clk_per_block = 256.0;
       const double fixed = 3000.0 + mb * 128.0 * p.r_cta * 4.0 / 128.0;
-      const int max_s = p.k_blocks < 256 ? p.k_blocks : 256;
+      const int max_s = single_split ? 1 : (p.k_blocks < 256 ? p.k_blocks : 256);
       for (int s = 1; s <= max_s; ++s) {
         const int64_t ctas = tiles * s;
         const int64_t waves = (ctas + kSmCount - 1) / kSmCount;
@@ -170,14 +170,22 @@ int launch_tc(int MB, int nslab, bool pair, dim3 grid, size_t smem, cudaStream_t
   return GRASS_ERR_UNSUPPORTED;
 }
 
+size_t norm_part_bytes(int64_t m, int64_t n) {
+  return round_up(static_cast<size_t>((n + 31) / 32) * round_up(static_cast<size_t>(m), 32) *
+                      sizeof(float), 256);
+}
+
+// norms != NULL: row-norm mode (idx NULL, r == m): the GEMM's epilogue reduces squares instead
+// of storing the gradient, then norms_finalize_kernel adds the per-column-group partials.
 int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T, int64_t m,
                  int64_t n, const int32_t* idx, const float* rho, int r, float* Gc, int64_t ldgc,
-                 void* ws, size_t ws_bytes, cudaStream_t s) {
+                 float* norms, void* ws, size_t ws_bytes, cudaStream_t s) {
   if (!aligned_to(X, 16) || ldx % 8 != 0) return GRASS_ERR_ALIGNMENT;
   if (idx == nullptr && (!aligned_to(dY, 16) || lddy % 8 != 0)) return GRASS_ERR_ALIGNMENT;
-  const TcPlan plan = make_plan(T, n, r);
+  const TcPlan plan = make_plan(T, n, r, norms != nullptr);
   const bool gather = idx != nullptr;
-  const size_t need = (gather ? plan.ag_bytes : 0) + plan.part_bytes;
+  const size_t need = norms != nullptr ? norm_part_bytes(m, n)
+                                       : (gather ? plan.ag_bytes : 0) + plan.part_bytes;
   if (need > 0 && (ws == nullptr || !aligned_to(ws, 256) || ws_bytes < need))
     return GRASS_ERR_WORKSPACE;
   cudaError_t err;
@@ -213,6 +221,8 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   p.k_blocks = plan.k_blocks;
   p.split_k = plan.split_k;
   p.status = status;
+  p.norm_part = norms != nullptr ? reinterpret_cast<float*>(wsp) : nullptr;
+  p.ld_norm = static_cast<long long>(round_up(static_cast<size_t>(m), 32));
   if (getenv("GRASS_DEBUG_PLAN") != nullptr)
     fprintf(stderr, "grass plan T=%lld n=%lld r=%d: r_cta=%d r_blocks=%d MB=%d n_blocks=%d "
                     "split_k=%d stages=%d pair=%d\n", static_cast<long long>(T), static_cast<long long>(n),
@@ -233,6 +243,13 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
             static_cast<unsigned>(plan.split_k));
   const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, grid, plan.smem_bytes, s, tmX, tmA, p);
   if (rc != GRASS_OK) return rc;
+  if (norms != nullptr) {
+    ProfileScope prof(GRASS_K_ROW_NORMS, s);
+    norms_finalize_kernel<<<static_cast<unsigned>((m + 255) / 256), 256, 0, s>>>(
+        p.norm_part, p.ld_norm, static_cast<int>((n + 31) / 32), static_cast<int>(m), norms);
+    GRASS_LAUNCH_CHECK();
+    return GRASS_OK;
+  }
   if (plan.split_k > 1) {
     const int vec = (n % 4 == 0) && (ldgc % 4 == 0) && aligned_to(Gc, 16);
     const long long work = static_cast<long long>(r) * (vec ? n / 4 : n);
@@ -272,7 +289,7 @@ extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, i
   if (r > m) return GRASS_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dt == GRASS_BF16)
-    return project_bf16(dY, lddy, X, ldx, T, m, n, idx, rho, r, Gc, ldgc, ws, ws_bytes, s);
+    return project_bf16(dY, lddy, X, ldx, T, m, n, idx, rho, r, Gc, ldgc, nullptr, ws, ws_bytes, s);
   if (dt != GRASS_F32) return GRASS_ERR_UNSUPPORTED;
   cudaError_t err;
   int* status = status_word(&err);
@@ -285,4 +302,34 @@ extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, i
       Gc, ldgc, status);
   GRASS_LAUNCH_CHECK();
   return GRASS_OK;
+}
+
+extern "C" size_t grass_grad_row_norms_workspace_bytes(int64_t T, int64_t m, int64_t n, int dt) {
+  (void)T;
+  if (m < 1 || n < 1) return 0;
+  if (dt == GRASS_BF16) return grass::norm_part_bytes(m, n) + 256;
+  return grass::round_up(static_cast<size_t>(m) * n * sizeof(float), 256) + 256;
+}
+
+extern "C" int grass_grad_row_norms(const void* dY, int64_t lddy, const void* X, int64_t ldx, int dt,
+                                    int64_t T, int64_t m, int64_t n, float* norms, void* ws,
+                                    size_t ws_bytes, void* stream) {
+  using namespace grass;
+  if (dY == nullptr || X == nullptr || norms == nullptr || T < 1 || m < 1 || n < 1 || lddy < m ||
+      ldx < n || T > 0x7fffffffLL || m > 0x7fffffffLL || n > 0x7fffffffLL)
+    return GRASS_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dt == GRASS_BF16)
+    return project_bf16(dY, lddy, X, ldx, T, m, n, nullptr, nullptr, static_cast<int>(m), nullptr,
+                        0, norms, ws, ws_bytes, s);
+  if (dt != GRASS_F32) return GRASS_ERR_UNSUPPORTED;
+  // fp32 path: the (small) gradient is formed in the workspace and reduced by grass_row_norms
+  if (ws == nullptr || !aligned_to(ws, 256) ||
+      ws_bytes < grass_grad_row_norms_workspace_bytes(T, m, n, dt) - 256)
+    return GRASS_ERR_WORKSPACE;
+  float* G = static_cast<float*>(ws);
+  const int rc = grass_project_grad(dY, lddy, X, ldx, dt, T, m, n, nullptr, nullptr,
+                                    static_cast<int32_t>(m), G, n, nullptr, 0, stream);
+  if (rc != GRASS_OK) return rc;
+  return grass_row_norms(G, GRASS_F32, m, n, n, norms, stream);
 }

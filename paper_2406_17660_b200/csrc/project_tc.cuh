@@ -65,8 +65,27 @@ struct TcParams {
   long long ld_out;     // row pitch of out, elements
   long long split_stride;  // elements between partials of consecutive splits
   const float* rho;     // applied here only when split_k == 1 (may be NULL)
+  float* norm_part;     // non-NULL: row-norm mode.  Nothing of D is stored; instead
+                        // norm_part[g * ld_norm + j] = sum of D[j, c]^2 over the 32 columns c of group g
+  long long ld_norm;
   int* status;
 };
+
+// Sum 32 per-lane values across the warp, all 32 at once: on return lane l holds
+// sum over lanes of x[l].  31 shuffles (halving exchange) instead of 32 x 5.
+__device__ __forceinline__ float warp_transpose_sum(float (&x)[32], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool upper = (lane & off) != 0;
+#pragma unroll
+    for (int k = 0; k < off; ++k) {
+      const float send = upper ? x[k] : x[k + off];
+      const float keep = upper ? x[k + off] : x[k];
+      x[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+  return x[0];
+}
 
 template <int MB, int NSLAB, bool PAIR>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -261,6 +280,16 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                                static_cast<uint32_t>(mb * R_CTA + j), v);
         ptx::tmem_ld_wait();
         const int c = c_base + mb * C_STEP + q * 32 + lane;
+        if (p.norm_part != nullptr) {
+          // fused row norms of the dense gradient (columns past n were zero-filled by TMA)
+          float sq[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) sq[i] = __uint_as_float(v[i]) * __uint_as_float(v[i]);
+          const float total = warp_transpose_sum(sq, lane);
+          const int g = (c_base + mb * C_STEP + q * 32) >> 5;
+          if (row0 + lane < p.r && (g << 5) < p.n) p.norm_part[g * p.ld_norm + row0 + lane] = total;
+          continue;
+        }
         float my_rho = 1.f;
         if (scale && row0 + lane < p.r) my_rho = __ldg(p.rho + row0 + lane);
         float* dst = out + static_cast<long long>(row0) * ld + c;
@@ -373,6 +402,17 @@ splitk_reduce_kernel(const float* __restrict__ part, long long ld_part, long lon
       Gc[static_cast<long long>(row) * ldgc + col] = acc * (rho != nullptr ? __ldg(rho + row) : 1.f);
     }
   }
+}
+
+// norms[j] = sqrt(sum over column groups g of part[g][j]), groups added in increasing g.
+__global__ void __launch_bounds__(256)
+norms_finalize_kernel(const float* __restrict__ part, long long ld, int groups, int m,
+                      float* __restrict__ norms) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= m) return;
+  float acc = 0.f;
+  for (int g = 0; g < groups; ++g) acc += part[g * ld + j];
+  norms[j] = sqrtf(acc);
 }
 
 }  // namespace grass

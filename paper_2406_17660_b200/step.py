@@ -15,22 +15,23 @@ from . import binding as B
 class GrassWorkspace:
     """Scratch shared by all layers of a model: sized for the largest layer.
 
-    Holds the m x n fp32 gradient used only on refresh iterations, the norms,
-    and the byte workspaces of grass_project_grad / grass_select.
+    Holds the norms and the byte workspaces of grass_project_grad,
+    grass_grad_row_norms and grass_select.  No m x n gradient buffer exists:
+    refresh iterations take the row norms straight from the GEMM's epilogue.
     """
 
     def __init__(self, shapes, T, r, dtype, method, device="cuda"):
         dt = B.BF16 if dtype == torch.bfloat16 else B.F32
-        max_mn = max(m * n for m, n in shapes)
         max_m = max(m for m, _ in shapes)
         proj = 256
         sel = 256
+        nrm = 256
         for m, n in shapes:
             rr = min(r, m)
-            proj = max(proj, B.grass_project_workspace_bytes(T, m, n, rr, dt),
-                       B.grass_project_workspace_bytes(T, m, n, m, dt))
+            proj = max(proj, B.grass_project_workspace_bytes(T, m, n, rr, dt))
+            nrm = max(nrm, B.grass_grad_row_norms_workspace_bytes(T, m, n, dt))
             sel = max(sel, B.grass_select_workspace_bytes(m, rr, method))
-        self.G = torch.empty(max_mn, dtype=torch.float32, device=device)
+        self.norm_ws = torch.empty(nrm, dtype=torch.uint8, device=device)
         self.norms = torch.empty(max_m, dtype=torch.float32, device=device)
         self.project_ws = torch.empty(proj, dtype=torch.uint8, device=device)
         self.select_ws = torch.empty(sel, dtype=torch.uint8, device=device)
@@ -61,10 +62,8 @@ class GrassLayer:
     def refresh(self, dY, X):
         """compute_P from this iteration's gradient (Algorithm 1, every K iterations)."""
         ws = self.ws
-        G = ws.G[: self.m * self.n].view(self.m, self.n)
-        B.grass_project_grad(dY, X, None, None, self.m, G, ws.project_ws)
         norms = ws.norms[: self.m]
-        B.grass_row_norms(G, norms)
+        B.grass_grad_row_norms(dY, X, norms, ws.norm_ws)
         B.grass_select(norms, self.r, self.method, self.seed, self.layer_id, self.t // self.K,
                        self.idx, self.rho, ws.select_ws)
         if self.reset_state:

@@ -57,6 +57,32 @@ def test_row_norms(m, n, ld, dtype):
     np.testing.assert_allclose(f64(norms), want, rtol=1e-5, atol=0)
 
 
+@pytest.mark.parametrize("T,m,n,dtype,ld", [
+    (512, 256, 256, torch.float32, None),
+    (100, 50, 70, torch.float32, None),
+    (1024, 512, 512, torch.bfloat16, None),
+    (777, 1376, 520, torch.bfloat16, None),              # 3 row blocks, ragged T
+    (640, 300, 328, torch.bfloat16, None),               # ragged m and n
+    (512, 2048, 5461, torch.bfloat16, 5464),             # padded pitch, n not a tile multiple
+    (256, 13824, 640, torch.bfloat16, None),             # 27 row blocks
+])
+def test_grad_row_norms_without_forming_the_gradient(T, m, n, dtype, ld):
+    X = syn.make_X(T, n, dtype, seed0=T + m)
+    dY = syn.make_dY(T, m, dtype, seed0=T + m)
+    Xd = syn._padded(X.to(DEV), ld or n)
+    norms = torch.full((m,), -1.0, dtype=torch.float32, device=DEV)
+    dt = grass.BF16 if dtype == torch.bfloat16 else grass.F32
+    ws = ws_bytes(grass.grass_grad_row_norms_workspace_bytes(T, m, n, dt))
+    dYd = syn._padded(dY.to(DEV), syn.pad_to(m, 8))      # the TMA path reads dY rows directly
+    grass.grass_grad_row_norms(dYd, Xd, norms, ws)
+    grass.grass_device_status()
+    want = oracle.grad_row_norms(f64(dY), f64(X))
+    np.testing.assert_allclose(f64(norms), want, rtol=1e-5)
+    again = torch.empty_like(norms)
+    grass.grass_grad_row_norms(dYd, Xd, again, ws)
+    assert torch.equal(again, norms)                      # fixed summation order
+
+
 # --------------------------------------------------------------------------- selection
 def _gpu_select(norms_np, r, method, seed=0, layer_id=0, epoch=0):
     norms = torch.tensor(norms_np, dtype=torch.float32, device=DEV)
