@@ -340,3 +340,38 @@ def layer_steps(W, batches, r, method, K, alpha, lr, beta1, beta2, eps,
                               Gc=Gc, M=M.copy(), V=V.copy(), U=U, W=W.copy(),
                               adam_step=adam_step))
     return W, M, V, sigma, rho
+
+
+# --------------------------------------------------------------------------
+# Projecting the smaller dimension (Section 4.1: "P is applied to project the
+# smaller dimension of G_W")
+# --------------------------------------------------------------------------
+def scatter_update_cols(W, U, sigma, rho, alpha, w_is_bf16=False):
+    """Column form of the apply step: W <- W + alpha * Delta P^T with P in R^{n x r}
+    selecting columns: W[:, sigma_j] += alpha * rho_j * U[j, :], U being r x m."""
+    W = np.array(W, dtype=np.float64, copy=True)
+    U = np.asarray(U, dtype=np.float64)
+    sigma = np.asarray(sigma, dtype=np.int64)
+    r = sigma.shape[0]
+    rho = np.ones(r) if rho is None else np.asarray(rho, dtype=np.float64)
+    for j in range(r):
+        W[:, sigma[j]] += alpha * rho[j] * U[j, :]
+    if w_is_bf16:
+        touched = np.unique(sigma)
+        W[:, touched] = round_to_bf16(W[:, touched])
+    return W
+
+
+def layer_steps_cols(W, batches, r, method, K, alpha, lr, beta1, beta2, eps, **kw):
+    """Algorithm 1 with the projection on the input dimension n (used when m > n):
+    G_C = G_W P is m x r, kept here as its transpose (r x m).  Selecting columns of
+    G_W = dY^T X is selecting rows of G_W^T = X^T dY, so this is Algorithm 1 on W^T
+    with the roles of dY and X exchanged."""
+    swapped = [(X, dY) for dY, X in batches]
+    trace = kw.get("trace")
+    Wt, M, V, sigma, rho = layer_steps(np.asarray(W, dtype=np.float64).T, swapped, r, method, K,
+                                       alpha, lr, beta1, beta2, eps, **kw)
+    if trace is not None:
+        for rec in trace:
+            rec["W"] = rec["W"].T
+    return Wt.T, M, V, sigma, rho

@@ -354,3 +354,38 @@ def test_without_replacement_matches_sequential_sampling_exactly_in_distribution
     with pytest.raises(oracle.DegenerateNorms):
         oracle.select(np.array([1.0, 0.0, 0.0]), 2, oracle.MULTINOMIAL_NORM_NR, seed=3)
     assert len(oracle.select(np.array([1.0, 0.0, 0.0]), 2, oracle.UNIFORM_NR, seed=3)[0]) == 2
+
+
+# ---- projecting the input dimension (Section 4.1, smaller-dimension rule) ----
+def test_column_projection_equals_dense_right_multiplication():
+    """G_C = G_W P, Adam on it, W += alpha * Delta P^T, written with dense matrices."""
+    rng = np.random.default_rng(12)
+    T, m, n, r = 7, 9, 5, 3
+    W0 = rng.standard_normal((m, n))
+    batches = [_small_problem(rng, T, m, n) for _ in range(4)]
+    hp = dict(lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8)
+    trace = []
+    oracle.layer_steps_cols(W0, batches, r, oracle.MULTINOMIAL_NORM, K=2, alpha=0.5,
+                            reset_state=True, seed=8, layer_id=1, trace=trace, **hp)
+    W = W0.copy()
+    for t, (dY, X) in enumerate(batches):
+        G = dY.T @ X                                              # m x n
+        if t % 2 == 0:
+            col_norms = np.sqrt(np.sum(G * G, axis=0))
+            sigma, rho = oracle.select(col_norms, r, oracle.MULTINOMIAL_NORM, 8, 1, t // 2)
+            P = np.zeros((n, r))
+            P[sigma, np.arange(r)] = rho
+            M, V = np.zeros((m, r)), np.zeros((m, r))
+            s = 0
+        s += 1
+        Mt, Vt, Ut = oracle.adam_update(M.T, V.T, (G @ P).T, hp["lr"], hp["beta1"], hp["beta2"],
+                                        hp["eps"], s)
+        M, V = Mt.T, Vt.T
+        W = W + 0.5 * Ut.T @ P.T
+        np.testing.assert_allclose(trace[t]["W"], W, rtol=1e-11, atol=1e-13)
+    U = rng.standard_normal((r, m))
+    sig = np.array([0, 3, 3])
+    rho3 = np.array([2.0, 0.5, 1.5])
+    out = oracle.scatter_update_cols(W0, U, sig, rho3, 0.25)
+    assert np.array_equal(out[:, [1, 2, 4]], W0[:, [1, 2, 4]])
+    np.testing.assert_allclose(out[:, 3], W0[:, 3] + 0.25 * (0.5 * U[1] + 1.5 * U[2]), rtol=1e-15)
