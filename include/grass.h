@@ -211,6 +211,20 @@ int grass_scatter_update(void* W, int wdt, int64_t m, int64_t n, int64_t ldw, co
                          double alpha, void* stream);
 
 /*
+ * Column form of the apply step, for layers projected on their input dimension
+ * (Section 4.1: P acts on the smaller dimension of the gradient, so for m > n
+ * the selection picks r of the n columns, G_C = G_W P, and W <- W + alpha U^T P^T):
+ *   W[c, idx_j] += alpha * rho_j * U[j, c],   c < m.
+ * U is r x m fp32 (the transpose of the m x r projected update, which is what
+ * grass_project_grad returns when it is called with dY and X exchanged: select
+ * columns of X, contract with dY).  idx ascending in [0, n), repeats adjacent and
+ * summed in fp32 in order of j, each element of W rounded once.
+ */
+int grass_scatter_update_cols(void* W, int wdt, int64_t m, int64_t n, int64_t ldw, const float* U,
+                              int64_t ldu, const int32_t* idx, const float* rho, int32_t r,
+                              double alpha, void* stream);
+
+/*
  * Read and clear the current device's status word.  Synchronises `stream`.
  * Returns GRASS_OK or the first error a kernel recorded since the last call;
  * if detail (host pointer, may be NULL) is given it receives a kernel-specific

@@ -49,6 +49,8 @@ _SIGNATURES = {
                                     c_int32, c_void_p]),
     "grass_scatter_update": (c_int, [c_void_p, c_int, c_int64, c_int64, c_int64, c_void_p, c_int64,
                                      c_void_p, c_void_p, c_int32, c_double, c_void_p]),
+    "grass_scatter_update_cols": (c_int, [c_void_p, c_int, c_int64, c_int64, c_int64, c_void_p,
+                                          c_int64, c_void_p, c_void_p, c_int32, c_double, c_void_p]),
     "grass_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int32)]),
     "grass_status_string": (ctypes.c_char_p, [c_int]),
     "grass_profile_begin": (c_int, [c_int32]),
@@ -207,6 +209,18 @@ def grass_scatter_update(W, U, idx, rho, alpha) -> None:
     _check(load_library().grass_scatter_update(_ptr(W), _dtype_code(W), m, n, _ld(W), _ptr(U),
                                                _ld(U), _ptr(idx), _ptr(rho), r, alpha, _stream()),
            "grass_scatter_update")
+
+
+def grass_scatter_update_cols(W, U, idx, rho, alpha) -> None:
+    m, n = W.shape
+    r = idx.numel()
+    _require(U, torch.float32, "U")
+    _require(idx, torch.int32, "idx")
+    if rho is not None:
+        _require(rho, torch.float32, "rho")
+    _check(load_library().grass_scatter_update_cols(_ptr(W), _dtype_code(W), m, n, _ld(W), _ptr(U),
+                                                    _ld(U), _ptr(idx), _ptr(rho), r, alpha,
+                                                    _stream()), "grass_scatter_update_cols")
 
 
 def grass_device_status(raise_on_error: bool = True):

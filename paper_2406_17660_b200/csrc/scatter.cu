@@ -98,6 +98,52 @@ scatter_kernel(T* __restrict__ W, int64_t m, int64_t n, int64_t ldw, const float
   }
 }
 
+// Column form (projection on the input dimension): W[c, idx_j] += alpha * rho_j * U[j, c].
+// A block owns 32 rows c of W and 32 consecutive j.  The U tile is read with c contiguous,
+// scaled, and transposed through shared memory; then lane l of a warp owns j = j0 + l, so the
+// 32 lanes touch 32 ascending columns of one W row (few sectors).  The first j of a run of
+// equal columns owns the column and adds the whole run (reaching past the tile through global
+// memory if the run does), so every element is rounded once.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+scatter_cols_kernel(T* __restrict__ W, int64_t m, int64_t n, int64_t ldw,
+                    const float* __restrict__ U, int64_t ldu, const int32_t* __restrict__ idx,
+                    const float* __restrict__ rho, int r, float alpha, int* status) {
+  __shared__ float tile[32][33];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t c0 = static_cast<int64_t>(blockIdx.x) * 32;
+  const int j0 = blockIdx.y * 32;
+  for (int jj = warp; jj < 32; jj += kThreads / 32) {
+    const int j = j0 + jj;
+    float v = 0.f;
+    if (j < r && c0 + lane < m)
+      v = alpha * (rho != nullptr ? rho[j] : 1.f) * U[static_cast<int64_t>(j) * ldu + c0 + lane];
+    tile[jj][lane] = v;
+  }
+  __syncthreads();
+  const int j = j0 + lane;
+  if (j >= r) return;
+  const int col = idx[j];
+  if (j > 0 && idx[j - 1] == col) return;              // not the head of its run
+  if (col < 0 || col >= n) {
+    if (blockIdx.x == 0 && warp == 0) record_status(status, GRASS_ERR_INVALID_ARG, col);
+    return;
+  }
+  int run = 1;
+  while (j + run < r && idx[j + run] == col) ++run;
+  for (int cc = warp; cc < 32; cc += kThreads / 32) {
+    const int64_t c = c0 + cc;
+    if (c >= m) break;
+    float acc = 0.f;
+    for (int k = 0; k < run; ++k) {
+      if (lane + k < 32) acc += tile[lane + k][cc];
+      else acc += alpha * (rho != nullptr ? rho[j + k] : 1.f) * U[static_cast<int64_t>(j + k) * ldu + c];
+    }
+    T* w = W + c * ldw + col;
+    *w = WTraits<T>::add1(*w, acc);
+  }
+}
+
 template <typename T>
 int launch(void* W, int64_t m, int64_t n, int64_t ldw, const float* U, int64_t ldu,
            const int32_t* idx, const float* rho, int r, float alpha, cudaStream_t s) {
@@ -136,4 +182,29 @@ extern "C" int grass_scatter_update(void* W, int wdt, int64_t m, int64_t n, int6
   if (wdt == GRASS_BF16)
     return grass::launch<__nv_bfloat16>(W, m, n, ldw, U, ldu, idx, rho, r, a, s);
   return GRASS_ERR_UNSUPPORTED;
+}
+
+extern "C" int grass_scatter_update_cols(void* W, int wdt, int64_t m, int64_t n, int64_t ldw,
+                                         const float* U, int64_t ldu, const int32_t* idx,
+                                         const float* rho, int32_t r, double alpha, void* stream) {
+  using namespace grass;
+  if (W == nullptr || U == nullptr || idx == nullptr || m < 1 || n < 1 || r < 1 || ldw < n ||
+      ldu < m || r > 65535 * 32 || n > 0x7fffffffLL)
+    return GRASS_ERR_INVALID_ARG;
+  if (wdt != GRASS_F32 && wdt != GRASS_BF16) return GRASS_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t err;
+  int* status = status_word(&err);
+  if (status == nullptr) GRASS_CUDA_TRY(err);
+  dim3 grid(static_cast<unsigned>((m + 31) / 32), static_cast<unsigned>((r + 31) / 32));
+  const float a = static_cast<float>(alpha);
+  ProfileScope prof(GRASS_K_SCATTER, s);
+  if (wdt == GRASS_F32)
+    scatter_cols_kernel<float><<<grid, kThreads, 0, s>>>(static_cast<float*>(W), m, n, ldw, U, ldu,
+                                                         idx, rho, r, a, status);
+  else
+    scatter_cols_kernel<__nv_bfloat16><<<grid, kThreads, 0, s>>>(
+        static_cast<__nv_bfloat16*>(W), m, n, ldw, U, ldu, idx, rho, r, a, status);
+  GRASS_LAUNCH_CHECK();
+  return GRASS_OK;
 }

@@ -41,9 +41,14 @@ class GrassLayer:
     """State of one linear layer W (m x n) trained by GRASS with rank r."""
 
     def __init__(self, W, r, method, K, alpha, lr, beta1=0.9, beta2=0.999, eps=1e-8,
-                 reset_state=True, seed=0, layer_id=0, workspace=None):
+                 reset_state=True, seed=0, layer_id=0, workspace=None, side="rows"):
+        """side = "rows": P selects r of the m output features (rows of W).
+        side = "cols": P selects r of the n input features (columns of W), the paper's choice
+        when m > n; the same library calls are used with dY and X exchanged, the state is
+        r x m, and the apply step is the column form."""
         self.W = W
-        self.m, self.n = W.shape
+        self.side = side
+        self.m, self.n = W.shape if side == "rows" else (W.shape[1], W.shape[0])
         self.r, self.method, self.K = r, method, K
         self.alpha, self.lr, self.beta1, self.beta2, self.eps = alpha, lr, beta1, beta2, eps
         self.reset_state, self.seed, self.layer_id = reset_state, seed, layer_id
@@ -73,11 +78,16 @@ class GrassLayer:
 
     def step(self, dY, X):
         """One iteration of Algorithm 1 for this layer; dY (T x m), X (T x n) on the device."""
+        if self.side == "cols":
+            dY, X = X, dY        # select columns of X, contract with dY: G_C^T = P^T (X^T dY)
         if self.t % self.K == 0:
             self.refresh(dY, X)
         self.adam_step += 1
         B.grass_project_grad(dY, X, self.idx, self.rho, self.r, self.Gc, self.ws.project_ws)
         B.grass_subspace_adam(self.Gc, self.M, self.V, self.U, self.lr, self.beta1, self.beta2,
                               self.eps, self.adam_step)
-        B.grass_scatter_update(self.W, self.U, self.idx, self.rho, self.alpha)
+        if self.side == "cols":
+            B.grass_scatter_update_cols(self.W, self.U, self.idx, self.rho, self.alpha)
+        else:
+            B.grass_scatter_update(self.W, self.U, self.idx, self.rho, self.alpha)
         self.t += 1

@@ -399,3 +399,66 @@ def test_layer_steps_bf16_multinomial_with_refresh():
 def test_layer_steps_bf16_topr_reset():
     _run_layer(1376, 512, 1024, 128, torch.bfloat16, grass.SEL_TOPR, K=2, steps=3, alpha=0.25,
                reset=True, seed=4)
+
+
+# --------------------------------------------------------------------------- column projection
+@pytest.mark.parametrize("m,n,ld,r,dtype", [
+    (300, 256, 256, 64, torch.float32), (1376, 512, 512, 128, torch.bfloat16),
+    (100, 77, 80, 40, torch.bfloat16), (64, 40, 40, 40, torch.float32),
+])
+def test_scatter_update_cols(m, n, ld, r, dtype):
+    rng = np.random.default_rng(m + n + r)
+    W = syn.make_W(m, n, dtype, seed0=r)
+    U = torch.tensor(rng.standard_normal((r, m)) * 1e-3, dtype=torch.float32)
+    sigma = np.sort(rng.choice(n, r, replace=True))          # repeats, some runs longer than a tile
+    sigma[: min(r, 36)] = sigma[0]
+    sigma = np.sort(sigma)
+    rho = (0.5 + 3 * rng.random(r)).astype(np.float32)
+    Wd = syn._padded(W.to(DEV), ld)
+    before = Wd.clone()
+    grass.grass_scatter_update_cols(Wd, U.to(DEV), torch.tensor(sigma, dtype=torch.int32, device=DEV),
+                                    torch.tensor(rho, device=DEV), 0.25)
+    grass.grass_device_status()
+    is_bf16 = dtype == torch.bfloat16
+    want = oracle.scatter_update_cols(f64(W), f64(U), sigma, rho, 0.25, w_is_bf16=is_bf16)
+    got = f64(Wd)
+    untouched = np.setdiff1d(np.arange(n), sigma)
+    assert torch.equal(Wd[:, untouched], before[:, untouched])
+    touched = np.unique(sigma)
+    if is_bf16:
+        exact = oracle.scatter_update_cols(f64(W), f64(U), sigma, rho, 0.25)[:, touched]
+        ulp = np.ldexp(1.0, np.floor(np.log2(np.maximum(np.abs(exact), 2.0 ** -126))).astype(int) - 7)
+        diff = np.abs(got[:, touched] - want[:, touched])
+        assert np.all(diff <= ulp * 1.0001) and np.mean(diff > 0) < 0.01
+    else:
+        np.testing.assert_allclose(got[:, touched], want[:, touched], rtol=1e-5, atol=1e-9)
+
+
+def test_layer_steps_projecting_the_input_dimension():
+    """gate/up-shaped layer (m > n): the selection picks input features (columns of W)."""
+    m, n, T, r = 1376, 512, 1024, 128
+    dtype, method = torch.bfloat16, grass.SEL_MULTINOMIAL_NORM
+    lr, b1, b2, eps = 1e-3, 0.9, 0.999, 1e-8
+    W = syn.make_W(m, n, dtype, seed0=8)
+    batches = [(syn.make_dY(T, m, dtype, seed0=8, step=t), syn.make_X(T, n, dtype, seed0=8, step=t))
+               for t in range(3)]
+    ws = grass.step.GrassWorkspace([(n, m)], T, r, dtype, method)
+    layer = grass.GrassLayer(W.to(DEV).clone(), r, method, 2, 0.25, lr, b1, b2, eps, reset_state=True,
+                             seed=8, layer_id=1, workspace=ws, side="cols")
+    trace = []
+    oracle.layer_steps_cols(f64(W), [(f64(a), f64(b)) for a, b in batches], r, method, 2, 0.25, lr,
+                            b1, b2, eps, reset_state=True, seed=8, layer_id=1, w_is_bf16=True,
+                            trace=trace)
+    for t, (dY, X) in enumerate(batches):
+        before = layer.W.clone()
+        layer.step(dY.to(DEV), X.to(DEV))
+        grass.grass_device_status()
+        ref = trace[t]
+        assert np.array_equal(layer.idx.cpu().numpy(), ref["sigma"])
+        assert layer.Gc.shape == (r, m) and rel_fro(f64(layer.Gc), ref["Gc"]) <= 1e-4
+        assert rel_fro(f64(layer.M), ref["M"]) <= 1e-4
+        untouched = np.setdiff1d(np.arange(n), ref["sigma"])
+        assert torch.equal(layer.W[:, untouched], before[:, untouched])
+        got = f64(layer.W)
+        assert np.max(np.abs(got - ref["W"])) <= 2.0 ** -7 * np.max(np.abs(ref["W"]))
+        assert np.mean(got != ref["W"]) < 0.02
