@@ -266,7 +266,8 @@ def run_gpu(args):
         W = syn.make_W(m, n, wl.dtype, layer=li, proj=pi, device=dev, ld=syn.pad_to(n, 8))
         layer = GrassLayer(W, min(wl.r, m), wl.method, K, wl.alpha, wl.lr, wl.beta1, wl.beta2,
                            wl.eps, reset_state=wl.reset_state, seed=0,
-                           layer_id=li * len(wl.shapes) + pi, workspace=wss[i % n_streams])
+                           layer_id=li * len(wl.shapes) + pi, workspace=wss[i % n_streams],
+                           fused_update=not args.unfused, keep_U=False)
         layer.stream = streams[i % n_streams]
         layers.append((pi, layer))
     in_bytes = sum(d.numel() * d.element_size() + x.numel() * x.element_size() for d, x in block_in)
@@ -370,9 +371,11 @@ def run_gpu(args):
         if "scatter" in per_kernel:
             b = (4.0 + 2 * wbytes) * rn * args.steps
             hbm["scatter"] = {"gbs": b / (per_kernel["scatter"]["ms"] * 1e-3) / 1e9}
-        if "row_norms" in per_kernel:
-            b = 4.0 * sum(m * n for _, m, n in wl.shapes) * wl.layers * len(refresh_steps)
-            hbm["row_norms"] = {"gbs": b / (per_kernel["row_norms"]["ms"] * 1e-3) / 1e9}
+        if "adam_scatter" in per_kernel:
+            b = (20.0 + 2 * wbytes) * rn * args.steps      # g, M, V in; M, V out; W in and out
+            hbm["adam_scatter"] = {"gbs": b / (per_kernel["adam_scatter"]["ms"] * 1e-3) / 1e9}
+        # (the step takes its row norms from the GEMM epilogue; the stand-alone row-norm kernel's
+        # bandwidth is measured by profile_case, see profiles/)
         for v in hbm.values():
             v["frac_of_hbm_peak"] = v["gbs"] / peaks["hbm_gbs"]
 
@@ -386,7 +389,10 @@ def run_gpu(args):
             hd.copy_(dY)
             hx.copy_(X)
             host_in.append((hd, hx))
-        stage = [(torch.empty_like(d), torch.empty_like(x)) for d, x in block_in]
+        def like(t):      # same shape AND row pitch (empty_like would drop the padding)
+            return torch.empty((t.shape[0], t.stride(0)), dtype=t.dtype, device=t.device)[:, : t.shape[1]]
+
+        stage = [(like(d), like(x)) for d, x in block_in]
         max_rn = max(l.Gc.numel() for _, l in layers)
         host_out = [torch.empty(max_rn, dtype=torch.float32, pin_memory=True) for _ in wl.shapes]
         e2e_steps = min(args.steps, args.e2e_steps)
@@ -482,6 +488,7 @@ def main():
     ap.add_argument("--refresh-every", type=int, default=None, help="override K")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--streams", type=int, default=2, help="streams that layers alternate over")
+    ap.add_argument("--unfused", action="store_true", help="separate Adam and apply kernels")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -211,6 +211,20 @@ int grass_scatter_update(void* W, int wdt, int64_t m, int64_t n, int64_t ldw, co
                          double alpha, void* stream);
 
 /*
+ * grass_subspace_adam followed by grass_scatter_update in one kernel (the two
+ * steps of Algorithm 1 after the projection; both are local to a selected row).
+ * Arguments as for the two calls; M and V are updated in place, W's selected rows
+ * are updated in place, and U is written only if it is not NULL (the update then
+ * never touches HBM: 24 bytes per element instead of 36).  Results are
+ * bit-identical to calling the two functions in turn.  idx ascending, repeats
+ * adjacent (every repeat keeps its own state row; the W row is written once).
+ */
+int grass_adam_scatter(const float* Gc, int64_t ldgc, float* M, float* V, float* U,
+                       int64_t ldstate, void* W, int wdt, int64_t m, int64_t n, int64_t ldw,
+                       const int32_t* idx, const float* rho, int32_t r, double lr, double beta1,
+                       double beta2, double eps, int32_t step, double alpha, void* stream);
+
+/*
  * Column form of the apply step, for layers projected on their input dimension
  * (Section 4.1: P acts on the smaller dimension of the gradient, so for m > n
  * the selection picks r of the n columns, G_C = G_W P, and W <- W + alpha U^T P^T):
@@ -254,7 +268,8 @@ typedef enum {
   GRASS_K_SPLITK_REDUCE = 4,
   GRASS_K_PROJECT_FP32 = 5,
   GRASS_K_ADAM = 6,
-  GRASS_K_SCATTER = 7
+  GRASS_K_SCATTER = 7,
+  GRASS_K_ADAM_SCATTER = 8   /* fused Adam + apply */
 } grass_kernel_t;
 int grass_profile_begin(int32_t max_launches);
 int grass_profile_end(int32_t* kernel_id, float* ms, int32_t* n_launches);

@@ -49,6 +49,10 @@ _SIGNATURES = {
                                     c_int32, c_void_p]),
     "grass_scatter_update": (c_int, [c_void_p, c_int, c_int64, c_int64, c_int64, c_void_p, c_int64,
                                      c_void_p, c_void_p, c_int32, c_double, c_void_p]),
+    "grass_adam_scatter": (c_int, [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int64, c_void_p,
+                                   c_int, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_int32,
+                                   c_double, c_double, c_double, c_double, c_int32, c_double,
+                                   c_void_p]),
     "grass_scatter_update_cols": (c_int, [c_void_p, c_int, c_int64, c_int64, c_int64, c_void_p,
                                           c_int64, c_void_p, c_void_p, c_int32, c_double, c_void_p]),
     "grass_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int32)]),
@@ -59,7 +63,7 @@ _SIGNATURES = {
 }
 
 KERNEL_NAMES = ["row_norms", "select", "gather", "project_tc", "splitk_reduce", "project_fp32",
-                "adam", "scatter"]
+                "adam", "scatter", "adam_scatter"]
 
 
 def load_library():
@@ -209,6 +213,25 @@ def grass_scatter_update(W, U, idx, rho, alpha) -> None:
     _check(load_library().grass_scatter_update(_ptr(W), _dtype_code(W), m, n, _ld(W), _ptr(U),
                                                _ld(U), _ptr(idx), _ptr(rho), r, alpha, _stream()),
            "grass_scatter_update")
+
+
+def grass_adam_scatter(Gc, M, V, U, W, idx, rho, lr, beta1, beta2, eps, step, alpha) -> None:
+    """Adam on the r x n state and the row-sparse apply in one kernel; U may be None."""
+    r, n = M.shape
+    m = W.shape[0]
+    for t, name in ((Gc, "Gc"), (M, "M"), (V, "V")):
+        _require(t, torch.float32, name)
+    if U is not None:
+        _require(U, torch.float32, "U")
+        if _ld(U) != _ld(M):
+            raise ValueError("M, V and U must share one row pitch")
+    if _ld(V) != _ld(M):
+        raise ValueError("M and V must share one row pitch")
+    _require(idx, torch.int32, "idx")
+    _check(load_library().grass_adam_scatter(_ptr(Gc), _ld(Gc), _ptr(M), _ptr(V), _ptr(U), _ld(M),
+                                             _ptr(W), _dtype_code(W), m, n, _ld(W), _ptr(idx),
+                                             _ptr(rho), r, lr, beta1, beta2, eps, step, alpha,
+                                             _stream()), "grass_adam_scatter")
 
 
 def grass_scatter_update_cols(W, U, idx, rho, alpha) -> None:

@@ -16,7 +16,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgrass_b200.so")
-SOURCES = ["common.cu", "row_norms.cu", "select.cu", "project.cu", "adam.cu", "scatter.cu"]
+SOURCES = ["common.cu", "row_norms.cu", "select.cu", "project.cu", "adam.cu", "scatter.cu",
+           "adam_scatter.cu"]
 
 
 def _nvcc() -> str:

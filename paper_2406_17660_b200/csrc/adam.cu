@@ -5,25 +5,10 @@
 // element, 128-bit accesses, no reuse.  The scalar factors (1 - beta, the
 // reciprocal bias corrections) are formed in double on the host and rounded
 // once to fp32.
-#include <math.h>
-
-#include "common.cuh"
+#include "update_common.cuh"
 
 namespace grass {
 namespace {
-
-struct AdamScalars {
-  float beta1, beta2, om_beta1, om_beta2, inv_bc1, inv_bc2, lr, eps;
-};
-
-__device__ __forceinline__ void adam_elem(float g, float& m, float& v, float& u,
-                                          const AdamScalars& a) {
-  m = a.beta1 * m + a.om_beta1 * g;
-  v = a.beta2 * v + a.om_beta2 * (g * g);
-  const float mhat = m * a.inv_bc1;
-  const float vhat = v * a.inv_bc2;
-  u = -a.lr * mhat / (sqrtf(vhat) + a.eps);
-}
 
 constexpr int kThreads = 256;
 
@@ -78,18 +63,8 @@ extern "C" int grass_subspace_adam(const float* Gc, int64_t ldgc, float* M, floa
   if (Gc == nullptr || M == nullptr || V == nullptr || U == nullptr || r < 1 || n < 1 ||
       ldgc < n || ldstate < n || step < 1)
     return GRASS_ERR_INVALID_ARG;
-  if (!(beta1 >= 0.0 && beta1 < 1.0 && beta2 >= 0.0 && beta2 < 1.0) || !(eps >= 0.0) ||
-      !isfinite(lr))
-    return GRASS_ERR_INVALID_ARG;
-  AdamScalars a;
-  a.beta1 = static_cast<float>(beta1);
-  a.beta2 = static_cast<float>(beta2);
-  a.om_beta1 = static_cast<float>(1.0 - beta1);
-  a.om_beta2 = static_cast<float>(1.0 - beta2);
-  a.inv_bc1 = static_cast<float>(1.0 / (1.0 - pow(beta1, static_cast<double>(step))));
-  a.inv_bc2 = static_cast<float>(1.0 / (1.0 - pow(beta2, static_cast<double>(step))));
-  a.lr = static_cast<float>(lr);
-  a.eps = static_cast<float>(eps);
+  if (!adam_args_ok(lr, beta1, beta2, eps, step)) return GRASS_ERR_INVALID_ARG;
+  const AdamScalars a = make_adam_scalars(lr, beta1, beta2, eps, step);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const bool vec = (n % 4 == 0) && (ldgc % 4 == 0) && (ldstate % 4 == 0) && aligned_to(Gc, 16) &&
                    aligned_to(M, 16) && aligned_to(V, 16) && aligned_to(U, 16);

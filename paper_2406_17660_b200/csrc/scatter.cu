@@ -5,41 +5,12 @@
 // idx is ascending, so repeated rows are adjacent.  The first j of each run of
 // equal rows owns the row: it sums alpha*rho_j*U[j,:] over its run in fp32, in
 // order of j, and writes the row once -- no atomics, bit-reproducible.
-#include "common.cuh"
+#include "update_common.cuh"
 
 namespace grass {
 namespace {
 
 constexpr int kThreads = 256;
-
-template <typename T> struct WTraits;
-template <> struct WTraits<float> {
-  static constexpr int N = 4;
-  using vec = float4;
-  static __device__ __forceinline__ void add_store(float* w, float4 v, const float* acc) {
-    v.x += acc[0]; v.y += acc[1]; v.z += acc[2]; v.w += acc[3];
-    *reinterpret_cast<float4*>(w) = v;
-  }
-  static __device__ __forceinline__ float add1(float w, float a) { return w + a; }
-};
-template <> struct WTraits<__nv_bfloat16> {
-  static constexpr int N = 8;
-  using vec = uint4;
-  static __device__ __forceinline__ void add_store(__nv_bfloat16* w, uint4 raw, const float* acc) {
-    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float2 f = __bfloat1622float2(h[i]);
-      f.x += acc[2 * i];
-      f.y += acc[2 * i + 1];
-      h[i] = __floats2bfloat162_rn(f.x, f.y);
-    }
-    *reinterpret_cast<uint4*>(w) = raw;
-  }
-  static __device__ __forceinline__ __nv_bfloat16 add1(__nv_bfloat16 w, float a) {
-    return __float2bfloat16_rn(__bfloat162float(w) + a);
-  }
-};
 
 template <typename T, bool VEC>
 __global__ void __launch_bounds__(kThreads)
@@ -77,11 +48,11 @@ scatter_kernel(T* __restrict__ W, int64_t m, int64_t n, int64_t ldw, const float
       }
 #pragma unroll
       for (int q = 0; q < N / 4; ++q) {
-        acc[0][4 * q + 0] += s * va[q].x; acc[0][4 * q + 1] += s * va[q].y;
-        acc[0][4 * q + 2] += s * va[q].z; acc[0][4 * q + 3] += s * va[q].w;
+        acc[0][4 * q + 0] = apply_acc(acc[0][4 * q + 0], s, va[q].x); acc[0][4 * q + 1] = apply_acc(acc[0][4 * q + 1], s, va[q].y);
+        acc[0][4 * q + 2] = apply_acc(acc[0][4 * q + 2], s, va[q].z); acc[0][4 * q + 3] = apply_acc(acc[0][4 * q + 3], s, va[q].w);
         if (two) {
-          acc[1][4 * q + 0] += s * vb[q].x; acc[1][4 * q + 1] += s * vb[q].y;
-          acc[1][4 * q + 2] += s * vb[q].z; acc[1][4 * q + 3] += s * vb[q].w;
+          acc[1][4 * q + 0] = apply_acc(acc[1][4 * q + 0], s, vb[q].x); acc[1][4 * q + 1] = apply_acc(acc[1][4 * q + 1], s, vb[q].y);
+          acc[1][4 * q + 2] = apply_acc(acc[1][4 * q + 2], s, vb[q].z); acc[1][4 * q + 3] = apply_acc(acc[1][4 * q + 3], s, vb[q].w);
         }
       }
     }
@@ -92,7 +63,7 @@ scatter_kernel(T* __restrict__ W, int64_t m, int64_t n, int64_t ldw, const float
     for (int64_t c = c0; c < c0 + N && c < n; ++c) {
       float acc = 0.f;
       for (int j = j0; j < r && idx[j] == row; ++j)
-        acc += alpha * (rho != nullptr ? rho[j] : 1.f) * U[static_cast<int64_t>(j) * ldu + c];
+        acc = apply_acc(acc, alpha * (rho != nullptr ? rho[j] : 1.f), U[static_cast<int64_t>(j) * ldu + c]);
       w[c] = WTraits<T>::add1(w[c], acc);
     }
   }

@@ -41,13 +41,17 @@ class GrassLayer:
     """State of one linear layer W (m x n) trained by GRASS with rank r."""
 
     def __init__(self, W, r, method, K, alpha, lr, beta1=0.9, beta2=0.999, eps=1e-8,
-                 reset_state=True, seed=0, layer_id=0, workspace=None, side="rows"):
+                 reset_state=True, seed=0, layer_id=0, workspace=None, side="rows",
+                 fused_update=True, keep_U=True):
         """side = "rows": P selects r of the m output features (rows of W).
         side = "cols": P selects r of the n input features (columns of W), the paper's choice
         when m > n; the same library calls are used with dY and X exchanged, the state is
         r x m, and the apply step is the column form."""
         self.W = W
         self.side = side
+        # rows only: Adam and the apply step in one kernel; keep_U=False also skips writing U
+        self.fused_update = fused_update and side == "rows"
+        self.keep_U = keep_U
         self.m, self.n = W.shape if side == "rows" else (W.shape[1], W.shape[0])
         self.r, self.method, self.K = r, method, K
         self.alpha, self.lr, self.beta1, self.beta2, self.eps = alpha, lr, beta1, beta2, eps
@@ -84,6 +88,12 @@ class GrassLayer:
             self.refresh(dY, X)
         self.adam_step += 1
         B.grass_project_grad(dY, X, self.idx, self.rho, self.r, self.Gc, self.ws.project_ws)
+        if self.fused_update:
+            B.grass_adam_scatter(self.Gc, self.M, self.V, self.U if self.keep_U else None, self.W,
+                                 self.idx, self.rho, self.lr, self.beta1, self.beta2, self.eps,
+                                 self.adam_step, self.alpha)
+            self.t += 1
+            return
         B.grass_subspace_adam(self.Gc, self.M, self.V, self.U, self.lr, self.beta1, self.beta2,
                               self.eps, self.adam_step)
         if self.side == "cols":

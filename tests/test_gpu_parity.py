@@ -462,3 +462,35 @@ def test_layer_steps_projecting_the_input_dimension():
         got = f64(layer.W)
         assert np.max(np.abs(got - ref["W"])) <= 2.0 ** -7 * np.max(np.abs(ref["W"]))
         assert np.mean(got != ref["W"]) < 0.02
+
+
+# --------------------------------------------------------------------------- fused Adam + apply
+@pytest.mark.parametrize("m,n,ld,r,dtype,step", [
+    (256, 256, 256, 32, torch.float32, 1), (512, 1376, 1376, 128, torch.bfloat16, 5),
+    (100, 37, 40, 9, torch.bfloat16, 2), (4096, 4096, 4096, 1024, torch.bfloat16, 3),
+])
+def test_fused_adam_scatter_is_bit_identical_to_the_two_calls(m, n, ld, r, dtype, step):
+    rng = np.random.default_rng(m + n + r)
+    g = torch.Generator().manual_seed(r + n)
+    Gc = (torch.randn((r, n), generator=g) * torch.exp(torch.randn((r, 1), generator=g))).to(DEV)
+    M0 = (torch.randn((r, n), generator=g) * 0.1).to(DEV)
+    V0 = (torch.rand((r, n), generator=g) * 0.01).to(DEV)
+    sigma = np.sort(rng.choice(m, r, replace=True))
+    idx = torch.tensor(sigma, dtype=torch.int32, device=DEV)
+    rho = torch.tensor((0.5 + rng.random(r)).astype(np.float32), device=DEV)
+    W0 = syn._padded(syn.make_W(m, n, dtype, seed0=r).to(DEV), ld)
+    hp = (1e-3, 0.9, 0.999, 1e-8)
+    M1, V1, U1, W1 = M0.clone(), V0.clone(), torch.empty_like(M0), W0.clone()
+    grass.grass_subspace_adam(Gc, M1, V1, U1, *hp, step)
+    grass.grass_scatter_update(W1, U1, idx, rho, 0.25)
+    for keep in (True, False):
+        M2, V2, W2 = M0.clone(), V0.clone(), W0.clone()
+        U2 = torch.full_like(M0, float("nan")) if keep else None
+        grass.grass_adam_scatter(Gc, M2, V2, U2, W2, idx, rho, *hp, step, 0.25)
+        grass.grass_device_status()
+        assert torch.equal(M2, M1) and torch.equal(V2, V1) and torch.equal(W2, W1)
+        if keep:
+            assert torch.equal(U2, U1)
+    # and against the oracle, through the two-call path already checked element by element above
+    Mo, Vo, Uo = oracle.adam_update(f64(M0), f64(V0), f64(Gc), *hp, step)
+    assert rel_fro(f64(M1), Mo) <= 1e-6 and rel_fro(f64(U1), Uo) <= 1e-5
