@@ -18,7 +18,7 @@ struct TcPlan {
   int r_cta, r_blocks;
   int MB, n_blocks;   // n_blocks = gridDim.x (CTAs, an even number when pair)
   bool pair;          // two CTAs share each MMA (cta_group::2)
-  int k_blocks, split_k, stages;
+  int k_blocks, split_k, stages, bk;   // bk: tokens per pipeline stage
   size_t smem_bytes;
   long long ld_part;        // pitch of a split-K partial, elements
   size_t ag_bytes, part_bytes;
@@ -36,7 +36,7 @@ TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false) {
   p.r_blocks = (r64 + 511) / 512;
   p.r_cta = static_cast<int>(round_up(static_cast<size_t>((r64 + p.r_blocks - 1) / p.r_blocks), 64));
   p.r_pad = p.r_cta * p.r_blocks;
-  p.k_blocks = static_cast<int>((T + kTcBK - 1) / kTcBK);
+  p.k_blocks = static_cast<int>((T + 31) / 32);   // in 32-token units while searching
   int mb_max = 512 / p.r_cta;
   mb_max = mb_max >= 4 ? 4 : (mb_max >= 2 ? 2 : 1);
   while (mb_max > 1 && static_cast<int64_t>(mb_max / 2) * 128 >= n) mb_max /= 2;  // not past n
@@ -80,6 +80,9 @@ TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false) {
     p.n_blocks = static_cast<int>((n + cta_cols - 1) / cta_cols) * (p.pair ? 2 : 1);
   }
   const int a_slabs = p.pair ? p.r_cta / 128 : p.r_cta / 64;
+  p.bk = tc_bk(p.MB, a_slabs);
+  p.k_blocks = static_cast<int>((T + p.bk - 1) / p.bk);
+  if (p.split_k > p.k_blocks) p.split_k = p.k_blocks;
   p.stages = tc_stages(p.MB, a_slabs);
   p.smem_bytes = static_cast<size_t>(p.stages) * tc_stage_bytes(p.MB, a_slabs) + 1024;
   p.ld_part = static_cast<long long>(round_up(static_cast<size_t>(n), 4));
@@ -102,13 +105,13 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   return fn;
 }
 
-// bf16 matrix [rows][cols] with row pitch ld (elements): box = {64 cols, 32 rows}, 128B swizzle.
-bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+// bf16 matrix [rows][cols] with row pitch ld (elements): box = {64 cols, bk rows}, 128B swizzle.
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int bk) {
   PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
   cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
-  cuuint32_t box[2] = {64, static_cast<cuuint32_t>(kTcBK)};
+  cuuint32_t box[2] = {64, static_cast<cuuint32_t>(bk)};
   cuuint32_t estr[2] = {1, 1};
   CUresult res = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -194,7 +197,7 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
 
   char* wsp = static_cast<char*>(ws);
   CUtensorMap tmX, tmA;
-  if (!make_map(&tmX, X, T, n, ldx)) return GRASS_ERR_CUDA;
+  if (!make_map(&tmX, X, T, n, ldx, plan.bk)) return GRASS_ERR_CUDA;
   if (gather) {
     __nv_bfloat16* Ag = reinterpret_cast<__nv_bfloat16*>(wsp);
     const __nv_bfloat16* dYb = static_cast<const __nv_bfloat16*>(dY);
@@ -208,10 +211,10 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
                                                           ni, Ag, status);
     }
     GRASS_LAUNCH_CHECK();
-    if (!make_map(&tmA, Ag, T, plan.r_pad, plan.r_pad)) return GRASS_ERR_CUDA;
+    if (!make_map(&tmA, Ag, T, plan.r_pad, plan.r_pad, plan.bk)) return GRASS_ERR_CUDA;
     wsp += plan.ag_bytes;
   } else {
-    if (!make_map(&tmA, dY, T, m, lddy)) return GRASS_ERR_CUDA;
+    if (!make_map(&tmA, dY, T, m, lddy, plan.bk)) return GRASS_ERR_CUDA;
   }
 
   TcParams p;

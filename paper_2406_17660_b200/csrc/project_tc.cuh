@@ -42,24 +42,34 @@
 
 namespace grass {
 
-constexpr int kTcBK = 32;                 // tokens per pipeline stage
-constexpr int kTcSlabBytes = kTcBK * 128; // [32 tokens][64 bf16]
+// Tokens per pipeline stage: 64 where at least four such stages fit, else 32.  A stage costs
+// the two issuing threads a fixed number of instructions (barrier wait, fence, commit, copy
+// issue); with 64 tokens that cost is spread over twice as many MMAs (234 -> 193 us on the
+// LLaMA-7B q shape).  A slab is [BK tokens][64 bf16].
 constexpr int kTcThreads = 320;
 constexpr int kTcMaxStages = 8;
 constexpr int kTcSmemBudget = 227 * 1024 - 1024;  // dynamic part; the rest holds the barriers
 constexpr long long kTcWaitLimit = 2000000000LL;  // SM clocks (~1 s)
 constexpr long long kTcDrainLimit = 200000000LL;  // give-up path: wait for work in flight
 
-__host__ __device__ constexpr int tc_stage_bytes(int MB, int NSLAB) { return (2 * MB + NSLAB) * kTcSlabBytes; }
-__host__ __device__ constexpr int tc_stages(int MB, int NSLAB) {
-  return (kTcSmemBudget - 1024) / tc_stage_bytes(MB, NSLAB) > kTcMaxStages
+__host__ __device__ constexpr int tc_stage_bytes_bk(int MB, int A_SLABS, int BK) {
+  return (2 * MB + A_SLABS) * BK * 128;
+}
+__host__ __device__ constexpr int tc_bk(int MB, int A_SLABS) {
+  return (kTcSmemBudget - 1024) / tc_stage_bytes_bk(MB, A_SLABS, 64) >= 4 ? 64 : 32;
+}
+__host__ __device__ constexpr int tc_stage_bytes(int MB, int A_SLABS) {
+  return tc_stage_bytes_bk(MB, A_SLABS, tc_bk(MB, A_SLABS));
+}
+__host__ __device__ constexpr int tc_stages(int MB, int A_SLABS) {
+  return (kTcSmemBudget - 1024) / tc_stage_bytes(MB, A_SLABS) > kTcMaxStages
              ? kTcMaxStages
-             : (kTcSmemBudget - 1024) / tc_stage_bytes(MB, NSLAB);
+             : (kTcSmemBudget - 1024) / tc_stage_bytes(MB, A_SLABS);
 }
 
 struct TcParams {
   int T, n, r;          // logical sizes
-  int k_blocks;         // ceil(T / 32)
+  int k_blocks;         // ceil(T / tokens per stage)
   int split_k;          // gridDim.z
   float* out;           // split_k == 1: Gc, else partials [split][r][ld_out]
   long long ld_out;     // row pitch of out, elements
@@ -95,6 +105,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   constexpr int X_SLABS = 2 * MB;
   constexpr int A_SLABS = PAIR ? NSLAB / 2 : NSLAB;   // slabs of the gathered operand this CTA stages
   constexpr int N_SLABS = X_SLABS + A_SLABS;
+  constexpr int kTcBK = tc_bk(MB, A_SLABS);           // tokens per stage
+  constexpr int kTcSlabBytes = kTcBK * 128;
   constexpr int STAGE_BYTES = tc_stage_bytes(MB, A_SLABS);
   constexpr int STAGES = tc_stages(MB, A_SLABS);
   constexpr int UMMA_M = PAIR ? 256 : 128;
