@@ -95,9 +95,13 @@ struct SelectArgs {
   double* cdf;    // [m]   (sampling methods)
   int* counts;    // [m]   (sampling methods)
   int* status;
+  int stage_norms;   // dynamic shared memory holds a copy of the norms (m floats) ...
+  int stage_counts;  // ... followed by the hit counters (m ints)
+  int stage_cdf;     // ... followed by the running sum (m doubles)
 };
 
 __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
+  extern __shared__ __align__(16) float s_dyn[];   // staged norms / scores, then hit counters
   __shared__ int s_hist[256];
   __shared__ int s_int[kWarps + 1];
   __shared__ double s_dbl[kWarps + 1];
@@ -111,10 +115,23 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
   if (tid == 0) s_flag = 0;
   __syncthreads();
   {
+    // the one pass that reads global memory: 8 loads in flight per thread, not one at a time
     int bad = 0;
-    for (int k = tid; k < m; k += kThreads) {
-      const float v = a.norms[k];
-      if (!(v >= 0.f) || isinf(v)) bad = k + 1;
+    for (int k0 = tid; k0 < m; k0 += 8 * kThreads) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int k = k0 + u * kThreads;
+        v[u] = k < m ? __ldg(a.norms + k) : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int k = k0 + u * kThreads;
+        if (k < m) {
+          if (a.stage_norms) s_dyn[k] = v[u];   // every later pass reads shared memory, not L2
+          if (!(v[u] >= 0.f) || isinf(v[u])) bad = k + 1;
+        }
+      }
     }
     if (bad) atomicMax(&s_flag, bad);
   }
@@ -124,12 +141,15 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
     return;
   }
 
-  const float* keys = a.norms;   // what the r largest are taken of
+  const float* nrm = a.stage_norms ? s_dyn : a.norms;
+  int* counts = a.stage_counts ? reinterpret_cast<int*>(s_dyn + ((m + 3) & ~3)) : a.counts;
+  double* cdf = a.stage_cdf ? reinterpret_cast<double*>(s_dyn + 2 * ((m + 3) & ~3)) : a.cdf;
+  const float* keys = nrm;   // what the r largest are taken of
   if (is_nr(a.method)) {
     // ---- without replacement: exponential race (Efraimidis & Spirakis).  Row k scores
     // w_k / (-log u_k), u_k = (word_k + 1/2) 2^-32; the r largest scores are distributed as r
     // successive draws without replacement.  Scores are rounded to fp32 and ranked as such. ----
-    float* scores = reinterpret_cast<float*>(a.cdf);
+    float* scores = a.stage_norms ? s_dyn : reinterpret_cast<float*>(a.cdf);   // in place if staged
     int positive = 0;
     for (int k = tid; k < m; k += kThreads) {
       const uint4 blk = philox4x32_10(make_uint4(static_cast<uint32_t>(k >> 2), a.layer_id, a.epoch,
@@ -138,7 +158,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
       const uint32_t sel = k & 3;
       const uint32_t word = sel == 0 ? blk.x : sel == 1 ? blk.y : sel == 2 ? blk.z : blk.w;
       const double u = (static_cast<double>(word) + 0.5) * 0x1p-32;
-      const double w = sampling_weight(a.method, a.norms[k]);
+      const double w = sampling_weight(a.method, nrm[k]);
       scores[k] = static_cast<float>(w / -log(u));
       positive += w > 0.0;
     }
@@ -162,65 +182,162 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
       const uint32_t himask = pass == 3 ? 0u : (0xffffffffu << (shift + 8));
       for (int k = tid; k < m; k += kThreads) {
         const uint32_t key = norm_key(keys[k]);
-        if ((key & himask) == prefix) atomicAdd(&s_hist[(key >> shift) & 0xff], 1);
+        // norms share their leading bytes, so most of a warp lands in one bin: one atomic per
+        // distinct bin per warp instead of one per row
+        const bool in = (key & himask) == prefix;
+        const uint32_t voters = __ballot_sync(__activemask(), in);
+        if (in) {
+          const uint32_t bin = (key >> shift) & 0xff;
+          const uint32_t peers = __match_any_sync(voters, bin);
+          if ((tid & 31) == __ffs(peers) - 1) atomicAdd(&s_hist[bin], __popc(peers));
+        }
       }
       __syncthreads();
-      if (tid == 0) {
-        int need = s_need, d = 255;
-        for (; d > 0; --d) {
-          if (s_hist[d] >= need) break;
-          need -= s_hist[d];
+      if (tid < 32) {
+        // digit d with (keys above d) < need <= (keys at or above d), found by one warp: lane l
+        // owns bins 8l..8l+7; a suffix scan over the lanes, then a look inside one lane's bins
+        int h[8], mine = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { h[i] = s_hist[8 * tid + i]; mine += h[i]; }
+        int incl = mine;                     // keys in this lane's bins and all higher lanes'
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int dn = __shfl_down_sync(0xffffffffu, incl, o);
+          if (tid + o < 32) incl += dn;
         }
-        s_need = need;                       // how many to take among keys with this digit
-        s_prefix = prefix | (static_cast<uint32_t>(d) << shift);
+        const int need = s_need;
+        const int above = incl - mine;       // keys in higher lanes' bins
+        const bool here = above < need && need <= incl;   // true in exactly one lane
+        if (here) {
+          int rem = need - above, d = 7;
+          for (; d > 0; --d) {
+            if (h[d] >= rem) break;
+            rem -= h[d];
+          }
+          s_need = rem;                      // how many to take among keys with this digit
+          s_prefix = prefix | (static_cast<uint32_t>(8 * tid + d) << shift);
+        }
       }
       __syncthreads();
     }
     const uint32_t tau = s_prefix;           // key of the r-th largest norm
     const int need_eq = s_need;              // rows equal to tau to take, lowest row first
-    // ---- emit in ascending row order ----
-    int eq_base = 0, out_base = 0;
-    for (int k0 = 0; k0 < m; k0 += kThreads) {
-      const int k = k0 + tid;
-      uint32_t key = 0u;
-      int is_eq = 0, is_gt = 0;
-      if (k < m) {
-        key = norm_key(keys[k]);
-        is_eq = key == tau;
-        is_gt = key > tau;
+    // ---- emit in ascending row order.  Each warp owns a contiguous segment of rows; one
+    // counting pass, one scan over the 32 warp totals, one writing pass: three block barriers
+    // in all, instead of a block-wide scan for every 1024 rows. ----
+    const int lane = tid & 31, warp = tid >> 5;
+    const int seg = ((m + kWarps - 1) / kWarps + 31) & ~31;   // rows per warp, multiple of 32
+    const int k_begin = warp * seg, k_end = k_begin + seg < m ? k_begin + seg : m;
+    int n_eq = 0, n_gt = 0;
+    for (int k0 = k_begin; k0 < k_end; k0 += 32) {
+      const int k = k0 + lane;
+      const uint32_t key = k < k_end ? norm_key(keys[k]) : 0u;
+      n_eq += __popc(__ballot_sync(0xffffffffu, k < k_end && key == tau));
+      n_gt += __popc(__ballot_sync(0xffffffffu, k < k_end && key > tau));
+    }
+    __shared__ int s_eq_base[kWarps], s_out_base[kWarps];
+    if (lane == 0) { s_eq_base[warp] = n_eq; s_out_base[warp] = n_gt; }
+    __syncthreads();
+    if (warp == 0) {
+      // exclusive prefix of the eq counts, then of the selected counts, over the 32 warps
+      const int eq = s_eq_base[lane], gt = s_out_base[lane];
+      int eq_incl = eq;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, eq_incl, o);
+        if (lane >= o) eq_incl += up;
       }
-      int eq_total, sel_total;
-      const int eq_incl = block_inclusive_scan<int>(is_eq, s_int, eq_total);
-      const int sel = is_gt || (is_eq && (eq_base + eq_incl - 1) < need_eq);
-      const int sel_incl = block_inclusive_scan<int>(sel, s_int, sel_total);
+      const int eq_excl = eq_incl - eq;
+      int take = need_eq - eq_excl;                    // equal rows this warp may still take
+      take = take < 0 ? 0 : (take > eq ? eq : take);
+      const int sel = gt + take;
+      int sel_incl = sel;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, sel_incl, o);
+        if (lane >= o) sel_incl += up;
+      }
+      s_eq_base[lane] = eq_excl;
+      s_out_base[lane] = sel_incl - sel;
+    }
+    __syncthreads();
+    int eq_base = s_eq_base[warp], out_base = s_out_base[warp];
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    for (int k0 = k_begin; k0 < k_end; k0 += 32) {
+      const int k = k0 + lane;
+      const uint32_t key = k < k_end ? norm_key(keys[k]) : 0u;
+      const bool is_eq = k < k_end && key == tau, is_gt = k < k_end && key > tau;
+      const uint32_t eq_bits = __ballot_sync(0xffffffffu, is_eq);
+      const bool sel = is_gt || (is_eq && eq_base + __popc(eq_bits & lt_mask) < need_eq);
+      const uint32_t sel_bits = __ballot_sync(0xffffffffu, sel);
       if (sel) {
-        const int pos = out_base + sel_incl - 1;
+        const int pos = out_base + __popc(sel_bits & lt_mask);
         a.idx[pos] = k;
         a.rho[pos] = 1.f;
       }
-      eq_base += eq_total;
-      out_base += sel_total;
+      eq_base += __popc(eq_bits);
+      out_base += __popc(sel_bits);
     }
     return;
   }
 
-  // ---- with replacement: inverse CDF of the sampling weights ----
-  double carry = 0.0;
-  for (int k0 = 0; k0 < m; k0 += kThreads) {
-    const int k = k0 + tid;
-    const double v = k < m ? sampling_weight(a.method, a.norms[k]) : 0.0;
-    double total;
-    const double incl = block_inclusive_scan<double>(v, s_dbl, total);
-    if (k < m) {
-      a.cdf[k] = carry + incl;
-      a.counts[k] = 0;
+  // ---- with replacement: inverse CDF of the sampling weights.  Same two-pass scheme as the
+  // emit above: a warp owns a contiguous segment of rows, sums it, one scan over the 32 warp
+  // totals gives every segment its base, and a second pass writes the running sum. ----
+  const int lane = tid & 31, warp = tid >> 5;
+  const int seg = ((m + kWarps - 1) / kWarps + 31) & ~31;
+  const int k_begin = warp * seg, k_end = k_begin + seg < m ? k_begin + seg : m;
+  __shared__ double s_wbase[kWarps];
+  __shared__ double s_total;
+  __shared__ int s_cbase[kWarps];
+  // local[k] = running sum inside the segment (warp scan per 32 rows, carried across the
+  // segment); cdf[k] = base[warp] + local[k] with base[w + 1] = base[w] + local total of w added
+  // by one thread in order, so the running sum is exactly monotone across segment borders and a
+  // draw can never land on a zero-weight row.
+  auto slice_scan = [&](int k0) {
+    const int k = k0 + lane;
+    double v = k < k_end ? sampling_weight(a.method, nrm[k]) : 0.0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const double up = __shfl_up_sync(0xffffffffu, v, o);
+      if (lane >= o) v += up;
     }
-    carry += total;
+    return v;
+  };
+  {
+    double run = 0.0;
+    for (int k0 = k_begin; k0 < k_end; k0 += 32)
+      run = run + __shfl_sync(0xffffffffu, slice_scan(k0), 31);
+    if (lane == 0) s_wbase[warp] = run;
   }
-  const double S = carry;
+  __syncthreads();
+  if (tid == 0) {
+    double base = 0.0;
+    for (int w = 0; w < kWarps; ++w) {
+      const double t = s_wbase[w];
+      s_wbase[w] = base;
+      base = base + t;
+    }
+    s_total = base;
+  }
+  __syncthreads();
+  const double S = s_total;
   if (!(S > 0.0)) {
     if (tid == 0) record_status(a.status, GRASS_ERR_DEGENERATE, -1);
     return;
+  }
+  {
+    const double base = s_wbase[warp];
+    double run = 0.0;
+    for (int k0 = k_begin; k0 < k_end; k0 += 32) {
+      const int k = k0 + lane;
+      const double v = slice_scan(k0);
+      if (k < k_end) {
+        cdf[k] = base + (run + v);
+        counts[k] = 0;
+      }
+      run = run + __shfl_sync(0xffffffffu, v, 31);
+    }
   }
   __syncthreads();  // cdf and counts visible block-wide (same CTA: global writes + barrier)
   for (int j = tid; j < r; j += kThreads) {
@@ -233,19 +350,47 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
     int lo = 0, hi = m - 1;                  // first k with cdf[k] > target
     while (lo < hi) {
       const int mid = (lo + hi) >> 1;
-      if (a.cdf[mid] > target) hi = mid; else lo = mid + 1;
+      if (cdf[mid] > target) hi = mid; else lo = mid + 1;
     }
-    atomicAdd(&a.counts[lo], 1);
+    atomicAdd(&counts[lo], 1);
   }
   __syncthreads();
-  int out_base = 0;
-  for (int k0 = 0; k0 < m; k0 += kThreads) {
-    const int k = k0 + tid;
-    const int cnt = k < m ? a.counts[k] : 0;
-    int total;
-    const int incl = block_inclusive_scan<int>(cnt, s_int, total);
+  // expand the hit counts in row order: per-warp totals, one scan, one writing pass
+  {
+    int run = 0;
+    for (int k0 = k_begin; k0 < k_end; k0 += 32) {
+      const int k = k0 + lane;
+      int c = k < k_end ? counts[k] : 0;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+      run += c;
+    }
+    if (lane == 0) s_cbase[warp] = run;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const int mine = s_cbase[lane];
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    s_cbase[lane] = incl - mine;
+  }
+  __syncthreads();
+  int out_base = s_cbase[warp];
+  for (int k0 = k_begin; k0 < k_end; k0 += 32) {
+    const int k = k0 + lane;
+    const int cnt = k < k_end ? counts[k] : 0;
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += up;
+    }
     if (cnt > 0) {
-      const double q = sampling_weight(a.method, a.norms[k]) / S;
+      const double q = sampling_weight(a.method, nrm[k]) / S;
       const float rho = static_cast<float>(1.0 / sqrt(static_cast<double>(r) * q));
       const int pos = out_base + incl - cnt;
       for (int i = 0; i < cnt; ++i) {
@@ -253,8 +398,33 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
         a.rho[pos + i] = rho;
       }
     }
-    out_base += total;
+    out_base += __shfl_sync(0xffffffffu, incl, 31);
   }
+}
+
+// Stage the norms (and, if they still fit, the hit counters) in shared memory: the kernel is a
+// chain of short passes over m values, each of which would otherwise wait on an L2 round trip.
+int launch_select(SelectArgs& a, cudaStream_t s) {
+  constexpr size_t kBudget = 200 * 1024;
+  const size_t m4 = (static_cast<size_t>(a.m) + 3) / 4 * 4 * sizeof(float);
+  a.stage_norms = m4 <= kBudget;
+  a.stage_counts = a.stage_norms && a.method != GRASS_SEL_TOPR && 2 * m4 <= kBudget;
+  a.stage_cdf = a.stage_counts && 4 * m4 <= kBudget;
+  const size_t smem = a.stage_norms ? (a.stage_cdf ? 4 * m4 : a.stage_counts ? 2 * m4 : m4) : 0;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  GRASS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+    GRASS_CUDA_TRY(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(kBudget)));
+    attr_set[dev] = true;
+  }
+  {
+    ProfileScope prof(GRASS_K_SELECT, s);
+    select_kernel<<<1, kThreads, smem, s>>>(a);
+  }
+  GRASS_LAUNCH_CHECK();
+  return GRASS_OK;
 }
 
 size_t cdf_bytes(int64_t m) { return round_up(static_cast<size_t>(m) * sizeof(double), 256); }
@@ -300,12 +470,7 @@ extern "C" int grass_select(const float* norms, int64_t m, int32_t r, int method
   a.epoch = epoch;
   a.idx = idx;
   a.rho = rho;
-  {
-    ProfileScope prof(GRASS_K_SELECT, static_cast<cudaStream_t>(stream));
-    select_kernel<<<1, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
-  }
-  GRASS_LAUNCH_CHECK();
-  return GRASS_OK;
+  return launch_select(a, static_cast<cudaStream_t>(stream));
 }
 
 // ---------------------------------------------------------------------------
@@ -376,7 +541,5 @@ extern "C" int grass_select_static(const float* norms, int64_t m, int32_t r, int
   // The kernel writes every running-sum entry it later reads and zeroes the
   // m hit counters before counting, so whatever an earlier call left in the
   // array is never observed.
-  select_kernel<<<1, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
-  GRASS_LAUNCH_CHECK();
-  return GRASS_OK;
+  return launch_select(a, static_cast<cudaStream_t>(stream));
 }

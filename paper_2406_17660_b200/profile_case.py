@@ -2,8 +2,8 @@
 
     python -m paper_2406_17660_b200.profile_case --op project --T 8192 --m 4096 --n 4096 --r 1024
 
-Ops: project (gather + tcgen05 GEMM + split-K reduce), dense (idx = NULL), adam, scatter, norms,
-select.  Prints the per-kernel event timings of the last repetition so that the plain run leaves a
+Ops: project (gather + tcgen05 GEMM + split-K reduce), dense (idx = NULL), gradnorms (dense GEMM
+with the row-norm epilogue), adam, scatter, fused (Adam + apply), norms, select (multinomial-norm) / selecttop / selectnr.  Prints the per-kernel event timings of the last repetition so that the plain run leaves a
 record next to the capture.
 """
 from __future__ import annotations
@@ -33,16 +33,19 @@ def main():
     idx = torch.sort(torch.randperm(a.m, device=dev)[:r]).values.to(torch.int32)
     rho = torch.ones(r, device=dev)
     Gc = torch.empty((r, a.n), dtype=torch.float32, device=dev)
-    if a.op in ("project", "dense"):
+    if a.op in ("project", "dense", "gradnorms"):
         X = syn.make_X(a.T, a.n, dt, device=dev, ld=syn.pad_to(a.n, 8))
         dY = syn.make_dY(a.T, a.m, dt, device=dev, ld=syn.pad_to(a.m, 8))
         ws = torch.empty(grass.grass_project_workspace_bytes(a.T, a.m, a.n, r, grass.BF16),
                          dtype=torch.uint8, device=dev)
+    if a.op == "gradnorms":
+        nws = torch.empty(grass.grass_grad_row_norms_workspace_bytes(a.T, a.m, a.n, grass.BF16),
+                          dtype=torch.uint8, device=dev)
     M = torch.zeros_like(Gc)
     V = torch.zeros_like(Gc)
     U = torch.empty_like(Gc)
     W = syn.make_W(a.m, a.n, dt, device=dev, ld=syn.pad_to(a.n, 8))
-    G = torch.randn((a.m, a.n), device=dev) if a.op in ("norms", "select") else None
+    G = torch.randn((a.m, a.n), device=dev) if a.op in ("norms", "select", "selecttop", "selectnr") else None
     norms = torch.empty(a.m, device=dev)
     sws = torch.empty(grass.grass_select_workspace_bytes(a.m, r, grass.SEL_MULTINOMIAL_NORM),
                       dtype=torch.uint8, device=dev)
@@ -56,13 +59,19 @@ def main():
             grass.grass_project_grad(dY, X, None, None, r, Gc, ws)
         elif a.op == "adam":
             grass.grass_subspace_adam(Gc, M, V, U, 1e-3, 0.9, 0.999, 1e-8, rep + 1)
+        elif a.op == "fused":
+            grass.grass_adam_scatter(Gc, M, V, None, W, idx, rho, 1e-3, 0.9, 0.999, 1e-8, rep + 1, 0.25)
+        elif a.op == "gradnorms":
+            grass.grass_grad_row_norms(dY, X, norms, nws)
         elif a.op == "scatter":
             grass.grass_scatter_update(W, Gc, idx, rho, 0.25)
         elif a.op == "norms":
             grass.grass_row_norms(G, norms)
-        elif a.op == "select":
+        elif a.op in ("select", "selecttop", "selectnr"):
+            method = {"select": grass.SEL_MULTINOMIAL_NORM, "selecttop": grass.SEL_TOPR,
+                      "selectnr": grass.SEL_MULTINOMIAL_NORM_NR}[a.op]
             grass.grass_row_norms(G, norms)
-            grass.grass_select(norms, r, grass.SEL_MULTINOMIAL_NORM, 0, 0, rep, idx, rho, sws)
+            grass.grass_select(norms, r, method, 0, 0, rep, idx, rho, sws)
         else:
             raise SystemExit(f"unknown op {a.op}")
         _, recs = grass.grass_profile_end()
