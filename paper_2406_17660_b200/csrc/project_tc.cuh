@@ -11,8 +11,8 @@
 // needs a transpose in HBM:  D^T[c, j] = sum_t X[t, c] * A[t, j]  with
 //   A-operand = X tile      (M = 128 columns of n, MN-major: c contiguous)
 //   B-operand = gathered dY (N = up to 256 selected rows, MN-major: j contiguous)
-// Both are staged by TMA as slabs of [32 tokens][64 elements] with the 128-byte
-// swizzle, which is the canonical MN-major UMMA layout.  TMEM lane = c, TMEM
+// Both are staged by TMA as slabs of [BK tokens][64 elements] (BK = 64 or 32)
+// with the 128-byte swizzle, which is the canonical MN-major UMMA layout.  TMEM lane = c, TMEM
 // column = j, so the epilogue's tcgen05.ld hands each warp 32 consecutive c for
 // one j per register: every store instruction writes 128 contiguous bytes.
 //
