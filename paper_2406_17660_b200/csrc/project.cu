@@ -180,6 +180,32 @@ size_t norm_part_bytes(int64_t m, int64_t n) {
 
 // norms != NULL: row-norm mode (idx NULL, r == m): the GEMM's epilogue reduces squares instead
 // of storing the gradient, then norms_finalize_kernel adds the per-column-group partials.
+// fp32 path: split the tokens when the output has too few 64 x 64 tiles to occupy the GPU.
+struct Fp32Plan {
+  int split;
+  int64_t tokens_per_split;
+  long long ld_part;
+  size_t part_bytes;
+};
+Fp32Plan make_fp32_plan(int64_t T, int64_t n, int r) {
+  Fp32Plan p;
+  const int64_t tiles = ((n + kSimtBC - 1) / kSimtBC) * ((r + kSimtBJ - 1) / kSimtBJ);
+  int64_t split = (2 * kSmCount + tiles - 1) / tiles;
+  const int64_t max_split = (T + 2 * kSimtBT - 1) / (2 * kSimtBT);   // at least 32 tokens a slice
+  if (split > max_split) split = max_split;
+  if (split > 64) split = 64;
+  if (split < 1) split = 1;
+  int64_t per = (T + split - 1) / split;
+  per = (per + kSimtBT - 1) / kSimtBT * kSimtBT;
+  p.tokens_per_split = per;
+  p.split = static_cast<int>((T + per - 1) / per);
+  p.ld_part = static_cast<long long>(round_up(static_cast<size_t>(n), 4));
+  p.part_bytes = p.split > 1
+                     ? round_up(static_cast<size_t>(p.split) * r * p.ld_part * sizeof(float), 256)
+                     : 0;
+  return p;
+}
+
 int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T, int64_t m,
                  int64_t n, const int32_t* idx, const float* rho, int r, float* Gc, int64_t ldgc,
                  float* norms, void* ws, size_t ws_bytes, cudaStream_t s) {
@@ -274,7 +300,7 @@ extern "C" size_t grass_project_workspace_bytes(int64_t T, int64_t m, int64_t n,
                                                 int dt) {
   (void)m;
   if (T < 1 || n < 1 || r < 1) return 0;
-  if (dt != GRASS_BF16) return 256;
+  if (dt != GRASS_BF16) return grass::make_fp32_plan(T, n, r).part_bytes + 256;
   const grass::TcPlan plan = grass::make_plan(T, n, r);
   return plan.ag_bytes + plan.part_bytes + 256;
 }
@@ -297,21 +323,39 @@ extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, i
   cudaError_t err;
   int* status = status_word(&err);
   if (status == nullptr) GRASS_CUDA_TRY(err);
+  const Fp32Plan fp = make_fp32_plan(T, n, r);
+  if (fp.split > 1 && (ws == nullptr || !aligned_to(ws, 256) || ws_bytes < fp.part_bytes))
+    return GRASS_ERR_WORKSPACE;
   dim3 grid(static_cast<unsigned>((n + kSimtBC - 1) / kSimtBC),
-            static_cast<unsigned>((r + kSimtBJ - 1) / kSimtBJ));
-  ProfileScope prof(GRASS_K_PROJECT_FP32, s);
-  project_simt_kernel<float><<<grid, kSimtThreads, 0, s>>>(
-      static_cast<const float*>(dY), lddy, static_cast<const float*>(X), ldx, T, m, n, idx, rho, r,
-      Gc, ldgc, status);
+            static_cast<unsigned>((r + kSimtBJ - 1) / kSimtBJ), static_cast<unsigned>(fp.split));
+  float* out = fp.split > 1 ? static_cast<float*>(ws) : Gc;
+  const int64_t ld_out = fp.split > 1 ? fp.ld_part : ldgc;
+  {
+    ProfileScope prof(GRASS_K_PROJECT_FP32, s);
+    project_simt_kernel<float><<<grid, kSimtThreads, 0, s>>>(
+        static_cast<const float*>(dY), lddy, static_cast<const float*>(X), ldx, T, m, n, idx, rho, r,
+        out, ld_out, fp.tokens_per_split, static_cast<int64_t>(r) * fp.ld_part, status);
+  }
   GRASS_LAUNCH_CHECK();
+  if (fp.split > 1) {
+    const int vec = (n % 4 == 0) && (ldgc % 4 == 0) && aligned_to(Gc, 16);
+    const long long work = static_cast<long long>(r) * (vec ? n / 4 : n);
+    long long blocks = (work + 255) / 256;
+    if (blocks > kSmCount * 8) blocks = kSmCount * 8;
+    ProfileScope prof(GRASS_K_SPLITK_REDUCE, s);
+    splitk_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(
+        out, fp.ld_part, static_cast<long long>(r) * fp.ld_part, fp.split, r, static_cast<int>(n),
+        rho, Gc, ldgc, vec);
+    GRASS_LAUNCH_CHECK();
+  }
   return GRASS_OK;
 }
 
 extern "C" size_t grass_grad_row_norms_workspace_bytes(int64_t T, int64_t m, int64_t n, int dt) {
-  (void)T;
-  if (m < 1 || n < 1) return 0;
+  if (m < 1 || n < 1 || T < 1) return 0;
   if (dt == GRASS_BF16) return grass::norm_part_bytes(m, n) + 256;
-  return grass::round_up(static_cast<size_t>(m) * n * sizeof(float), 256) + 256;
+  return grass::round_up(static_cast<size_t>(m) * n * sizeof(float), 256) +
+         grass::make_fp32_plan(T, n, static_cast<int>(m)).part_bytes + 256;
 }
 
 extern "C" int grass_grad_row_norms(const void* dY, int64_t lddy, const void* X, int64_t ldx, int dt,
@@ -331,8 +375,10 @@ extern "C" int grass_grad_row_norms(const void* dY, int64_t lddy, const void* X,
       ws_bytes < grass_grad_row_norms_workspace_bytes(T, m, n, dt) - 256)
     return GRASS_ERR_WORKSPACE;
   float* G = static_cast<float*>(ws);
+  const size_t g_bytes = round_up(static_cast<size_t>(m) * n * sizeof(float), 256);
   const int rc = grass_project_grad(dY, lddy, X, ldx, dt, T, m, n, nullptr, nullptr,
-                                    static_cast<int32_t>(m), G, n, nullptr, 0, stream);
+                                    static_cast<int32_t>(m), G, n, static_cast<char*>(ws) + g_bytes,
+                                    ws_bytes - g_bytes, stream);
   if (rc != GRASS_OK) return rc;
   return grass_row_norms(G, GRASS_F32, m, n, n, norms, stream);
 }

@@ -75,4 +75,4 @@ def test_workspace_queries_are_host_only_and_monotone(lib):
     big = binding.grass_project_workspace_bytes(32768, 4096, 4096, 1024, binding.BF16)
     assert 1024 * 128 * 2 <= small < big
     assert big >= 32768 * 1024 * 2
-    assert binding.grass_project_workspace_bytes(1024, 512, 512, 128, binding.F32) == 256
+    assert binding.grass_project_workspace_bytes(1024, 512, 512, 128, binding.F32) >= 256
