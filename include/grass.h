@@ -171,9 +171,11 @@ int grass_project_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx,
  * and the m x n matrix is never written.  Arguments as for grass_project_grad
  * with idx = NULL; norms [m] fp32 is written; ws needs
  * grass_grad_row_norms_workspace_bytes(T, m, n, dt) bytes (GRASS_BF16: m * n / 8
- * bytes of per-column-group partial sums, added in a fixed order; GRASS_F32: the
- * fp32 path forms the small gradient in ws and calls grass_row_norms).  The
- * token sum is not split, so every square is taken of a complete dot product.
+ * bytes of per-column-group partial sums, added in a fixed order; a gradient too
+ * small to occupy the GPU unsplit is instead summed over token slices in fp32
+ * scratch and reduced from there; GRASS_F32: the fp32 path forms the small
+ * gradient in ws and calls grass_row_norms).  Every square is taken of a complete
+ * dot product.
  */
 size_t grass_grad_row_norms_workspace_bytes(int64_t T, int64_t m, int64_t n, int dt);
 int grass_grad_row_norms(const void* dY, int64_t lddy, const void* X, int64_t ldx, int dt,

@@ -206,15 +206,27 @@ Fp32Plan make_fp32_plan(int64_t T, int64_t n, int r) {
   return p;
 }
 
+// Row-norm mode.  The squares must be taken of complete dot products, so the fused epilogue
+// needs an unsplit token sum; that is the plan whenever the dense m x n output has enough tiles
+// to occupy the GPU (every LLaMA shape from 1B up).  A small gradient (few tiles) would leave
+// most SMs idle, so it is computed with the usual token split into fp32 partials -- small by
+// the same token -- and splitk_rownorms_kernel sums, squares and reduces them.
+TcPlan make_norms_plan(int64_t T, int64_t n, int r) {
+  const TcPlan fused = make_plan(T, n, r, true);
+  if (static_cast<int64_t>(fused.n_blocks) * fused.r_blocks >= 120) return fused;
+  return make_plan(T, n, r, false);
+}
+
 int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T, int64_t m,
                  int64_t n, const int32_t* idx, const float* rho, int r, float* Gc, int64_t ldgc,
                  float* norms, void* ws, size_t ws_bytes, cudaStream_t s) {
   if (!aligned_to(X, 16) || ldx % 8 != 0) return GRASS_ERR_ALIGNMENT;
   if (idx == nullptr && (!aligned_to(dY, 16) || lddy % 8 != 0)) return GRASS_ERR_ALIGNMENT;
-  const TcPlan plan = make_plan(T, n, r, norms != nullptr);
+  const TcPlan plan = norms != nullptr ? make_norms_plan(T, n, r) : make_plan(T, n, r);
   const bool gather = idx != nullptr;
-  const size_t need = norms != nullptr ? norm_part_bytes(m, n)
-                                       : (gather ? plan.ag_bytes : 0) + plan.part_bytes;
+  const bool fused_norms = norms != nullptr && plan.split_k == 1;
+  const size_t need = fused_norms ? norm_part_bytes(m, n)
+                                  : (gather ? plan.ag_bytes : 0) + plan.part_bytes;
   if (need > 0 && (ws == nullptr || !aligned_to(ws, 256) || ws_bytes < need))
     return GRASS_ERR_WORKSPACE;
   cudaError_t err;
@@ -250,7 +262,7 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   p.k_blocks = plan.k_blocks;
   p.split_k = plan.split_k;
   p.status = status;
-  p.norm_part = norms != nullptr ? reinterpret_cast<float*>(wsp) : nullptr;
+  p.norm_part = fused_norms ? reinterpret_cast<float*>(wsp) : nullptr;
   p.ld_norm = static_cast<long long>(round_up(static_cast<size_t>(m), 32));
   if (getenv("GRASS_DEBUG_PLAN") != nullptr)
     fprintf(stderr, "grass plan T=%lld n=%lld r=%d: r_cta=%d r_blocks=%d MB=%d n_blocks=%d "
@@ -258,7 +270,7 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
             r, plan.r_cta, plan.r_blocks, plan.MB, plan.n_blocks, plan.split_k, plan.stages,
             plan.pair ? 1 : 0);
   if (plan.split_k == 1) {
-    p.out = Gc;
+    p.out = Gc;            // unused in row-norm mode
     p.ld_out = ldgc;
     p.split_stride = 0;
     p.rho = rho;
@@ -274,8 +286,13 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   if (rc != GRASS_OK) return rc;
   if (norms != nullptr) {
     ProfileScope prof(GRASS_K_ROW_NORMS, s);
-    norms_finalize_kernel<<<static_cast<unsigned>((m + 255) / 256), 256, 0, s>>>(
-        p.norm_part, p.ld_norm, static_cast<int>((n + 31) / 32), static_cast<int>(m), norms);
+    if (fused_norms)
+      norms_finalize_kernel<<<static_cast<unsigned>((m + 255) / 256), 256, 0, s>>>(
+          p.norm_part, p.ld_norm, static_cast<int>((n + 31) / 32), static_cast<int>(m), norms);
+    else
+      splitk_rownorms_kernel<<<static_cast<unsigned>(m), 256, 0, s>>>(
+          p.out, plan.ld_part, p.split_stride, plan.split_k, static_cast<int>(m),
+          static_cast<int>(n), norms);
     GRASS_LAUNCH_CHECK();
     return GRASS_OK;
   }
@@ -353,7 +370,10 @@ extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, i
 
 extern "C" size_t grass_grad_row_norms_workspace_bytes(int64_t T, int64_t m, int64_t n, int dt) {
   if (m < 1 || n < 1 || T < 1) return 0;
-  if (dt == GRASS_BF16) return grass::norm_part_bytes(m, n) + 256;
+  if (dt == GRASS_BF16) {
+    const grass::TcPlan plan = grass::make_norms_plan(T, n, static_cast<int>(m));
+    return (plan.split_k == 1 ? grass::norm_part_bytes(m, n) : plan.part_bytes) + 256;
+  }
   return grass::round_up(static_cast<size_t>(m) * n * sizeof(float), 256) +
          grass::make_fp32_plan(T, n, static_cast<int>(m)).part_bytes + 256;
 }

@@ -416,6 +416,39 @@ splitk_reduce_kernel(const float* __restrict__ part, long long ld_part, long lon
   }
 }
 
+// Row norms from split-K partials of a small dense gradient: norms[j] = sqrt(sum_c (sum_s
+// part[s][j][c])^2).  One CTA per row; splits added in increasing s (four loads in flight),
+// columns by a fixed thread-strided order, then a shuffle tree and one shared-memory hop:
+// bit-reproducible.
+__global__ void __launch_bounds__(256)
+splitk_rownorms_kernel(const float* __restrict__ part, long long ld_part, long long split_stride,
+                       int split_k, int m, int n, float* __restrict__ norms) {
+  __shared__ float s_part[8];
+  const int j = blockIdx.x;
+  const float* row = part + static_cast<long long>(j) * ld_part;
+  float acc = 0.f;
+  for (int c = threadIdx.x; c < n; c += 256) {
+    const float* p = row + c;
+    float g = 0.f;
+    int s = 0;
+    for (; s + 3 < split_k; s += 4) {
+      const float a0 = p[(s + 0) * split_stride], a1 = p[(s + 1) * split_stride],
+                  a2 = p[(s + 2) * split_stride], a3 = p[(s + 3) * split_stride];
+      g = (((g + a0) + a1) + a2) + a3;
+    }
+    for (; s < split_k; ++s) g += p[s * split_stride];
+    acc = fmaf(g, g, acc);
+  }
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float v = threadIdx.x < 8 ? s_part[threadIdx.x] : 0.f;
+    v = warp_sum(v);
+    if (threadIdx.x == 0) norms[j] = sqrtf(v);
+  }
+}
+
 // norms[j] = sqrt(sum over column groups g of part[g][j]), groups added in increasing g.
 __global__ void __launch_bounds__(256)
 norms_finalize_kernel(const float* __restrict__ part, long long ld, int groups, int m,
