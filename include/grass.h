@@ -251,6 +251,16 @@ int grass_device_status(void* stream, int32_t* detail);
 const char* grass_status_string(int status);
 
 /*
+ * Self-test of the bounded device-side wait (the paper has no counterpart).  Every
+ * mbarrier wait in the projection kernel gives up after a fixed number of SM clocks,
+ * records GRASS_ERR_TIMEOUT and lets the kernel return instead of spinning forever.
+ * This call launches one thread that waits on a barrier nothing completes, for at
+ * most limit_cycles (1 .. 2e9) clocks; afterwards grass_device_status reports
+ * GRASS_ERR_TIMEOUT with detail 900 and the context stays usable.
+ */
+int grass_selftest_bounded_wait(int64_t limit_cycles, void* stream);
+
+/*
  * Per-launch timing of the library's own kernels (a measurement aid; the paper
  * has no counterpart).  Between grass_profile_begin and grass_profile_end every
  * kernel the library launches on the calling thread's behalf is bracketed by a

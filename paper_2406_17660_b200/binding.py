@@ -57,6 +57,7 @@ _SIGNATURES = {
                                           c_int64, c_void_p, c_void_p, c_int32, c_double, c_void_p]),
     "grass_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int32)]),
     "grass_status_string": (ctypes.c_char_p, [c_int]),
+    "grass_selftest_bounded_wait": (c_int, [c_int64, c_void_p]),
     "grass_profile_begin": (c_int, [c_int32]),
     "grass_profile_end": (c_int, [ctypes.POINTER(c_int32), ctypes.POINTER(ctypes.c_float),
                                   ctypes.POINTER(c_int32)]),
@@ -253,6 +254,11 @@ def grass_device_status(raise_on_error: bool = True):
     if status != 0 and raise_on_error:
         raise GrassError(status, f"device status (detail {detail.value})")
     return status, detail.value
+
+
+def grass_selftest_bounded_wait(limit_cycles: int) -> None:
+    _check(load_library().grass_selftest_bounded_wait(limit_cycles, _stream()),
+           "grass_selftest_bounded_wait")
 
 
 def grass_profile_begin(max_launches: int) -> None:

@@ -17,7 +17,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgrass_b200.so")
 SOURCES = ["common.cu", "row_norms.cu", "select.cu", "project.cu", "adam.cu", "scatter.cu",
-           "adam_scatter.cu"]
+           "adam_scatter.cu", "selftest.cu"]
 
 
 def _nvcc() -> str:

@@ -494,3 +494,17 @@ def test_fused_adam_scatter_is_bit_identical_to_the_two_calls(m, n, ld, r, dtype
     # and against the oracle, through the two-call path already checked element by element above
     Mo, Vo, Uo = oracle.adam_update(f64(M0), f64(V0), f64(Gc), *hp, step)
     assert rel_fro(f64(M1), Mo) <= 1e-6 and rel_fro(f64(U1), Uo) <= 1e-5
+
+
+# --------------------------------------------------------------------------- bounded waits
+def test_a_wait_that_nothing_completes_times_out_and_leaves_the_context_usable():
+    grass.grass_device_status(raise_on_error=False)              # start from a clean status word
+    grass.grass_selftest_bounded_wait(1_000_000)                 # ~0.5 ms at 1.9 GHz
+    status, detail = grass.grass_device_status(raise_on_error=False)
+    assert status == 7 and detail == 900                         # GRASS_ERR_TIMEOUT
+    assert grass.grass_device_status(raise_on_error=False)[0] == 0   # reading clears it
+    G = torch.ones((4, 16), device=DEV)
+    norms = torch.empty(4, device=DEV)
+    grass.grass_row_norms(G, norms)                              # the GPU still does work
+    grass.grass_device_status()
+    assert torch.allclose(norms, torch.full((4,), 4.0, device=DEV))
