@@ -25,13 +25,16 @@ def f64(t):
     (32768, 4096, 4096, 1024, grass.SEL_TOPR),              # 7B q: CTA pairs, 2 row blocks, split-K 2
     (32768, 4096, 11008, 1024, grass.SEL_TOPR),             # 7B down: 86 n-tiles, split-K 4
     (65536, 1376, 512, 128, grass.SEL_MULTINOMIAL_NORM),    # 60M gate: 4 n-blocks per CTA, 64 splits
+    (32768, 13824, 5120, 1024, grass.SEL_TOPR),             # 13B gate: largest row count, sparse pick
+    (65536, 2048, 5461, 512, grass.SEL_MULTINOMIAL_NORM_NR),  # 1B down: padded pitch, no replacement
 ])
 def test_layer_step_on_sampled_rows(T, m, n, r, method):
     dt = torch.bfloat16
     X = syn.make_X(T, n, dt, seed0=11)
     dY = syn.make_dY(T, m, dt, seed0=11)
     W = syn.make_W(m, n, dt, seed0=11)
-    Xd, dYd = X.to(DEV), dY.to(DEV)
+    Xd = syn._padded(X.to(DEV), syn.pad_to(n, 8))            # 16-byte row pitch for the TMA path
+    dYd = syn._padded(dY.to(DEV), syn.pad_to(m, 8))
     ws = grass.step.GrassWorkspace([(m, n)], T, r, dt, method)
     layer = grass.GrassLayer(W.to(DEV).clone(), r, method, K=200, alpha=0.25, lr=1e-3,
                              reset_state=True, seed=5, layer_id=2, workspace=ws)
