@@ -300,7 +300,7 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
     const int vec = (n % 4 == 0) && (ldgc % 4 == 0) && aligned_to(Gc, 16);
     const long long work = static_cast<long long>(r) * (vec ? n / 4 : n);
     long long blocks = (work + 255) / 256;
-    if (blocks > kSmCount * 8) blocks = kSmCount * 8;
+    if (blocks > kSmCount * 32) blocks = kSmCount * 32;
     ProfileScope prof(GRASS_K_SPLITK_REDUCE, s);
     splitk_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(
         p.out, plan.ld_part, p.split_stride, plan.split_k, r, static_cast<int>(n), rho, Gc, ldgc,
@@ -358,7 +358,7 @@ extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, i
     const int vec = (n % 4 == 0) && (ldgc % 4 == 0) && aligned_to(Gc, 16);
     const long long work = static_cast<long long>(r) * (vec ? n / 4 : n);
     long long blocks = (work + 255) / 256;
-    if (blocks > kSmCount * 8) blocks = kSmCount * 8;
+    if (blocks > kSmCount * 32) blocks = kSmCount * 32;
     ProfileScope prof(GRASS_K_SPLITK_REDUCE, s);
     splitk_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(
         out, fp.ld_part, static_cast<long long>(r) * fp.ld_part, fp.split, r, static_cast<int>(n),

@@ -395,7 +395,18 @@ splitk_reduce_kernel(const float* __restrict__ part, long long ld_part, long lon
       const int row = static_cast<int>(i / nv), col = static_cast<int>(i - static_cast<long long>(row) * nv) * 4;
       const float* src = part + static_cast<long long>(row) * ld_part + col;
       float4 acc = *reinterpret_cast<const float4*>(src);
-      for (int s = 1; s < split_k; ++s) {
+      int s = 1;
+      for (; s + 3 < split_k; s += 4) {   // four loads in flight; the order of the adds is fixed
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          v[u] = *reinterpret_cast<const float4*>(src + (s + u) * split_stride);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w;
+        }
+      }
+      for (; s < split_k; ++s) {
         const float4 v = *reinterpret_cast<const float4*>(src + s * split_stride);
         acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
       }
