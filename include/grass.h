@@ -227,6 +227,35 @@ int grass_adam_scatter(const float* Gc, int64_t ldgc, float* M, float* V, float*
                        double beta2, double eps, int32_t step, double alpha, void* stream);
 
 /*
+ * The two per-step calls for up to 8 layers of one shape in a single set of
+ * launches (the paper applies the same step to every linear layer; the q, k, v, o
+ * projections of a block share a shape, as do gate and up).  Small layers are
+ * bound by per-launch costs and by split-K partial traffic; one launch over
+ * `count` layers has `count` times the tiles, so it needs a `count` times smaller
+ * token split.  Every array argument is a HOST array of `count` device pointers;
+ * layer g uses dY[g], X[g], idx[g] (required), rho[g] (the array or an entry may be
+ * NULL), Gc[g], and M[g], V[g], U[g] (array or entries may be NULL), W[g].  All
+ * layers share T, m, n, r, the pitches, the dtype (GRASS_BF16 for the projection)
+ * and the hyper-parameters.  Results are bit-identical to `count` separate
+ * bit-reproducible calls only where the token split is the same; in general they
+ * agree to fp32 summation order.  ws needs
+ * grass_project_batched_workspace_bytes(count, T, m, n, r) bytes.
+ */
+size_t grass_project_batched_workspace_bytes(int32_t count, int64_t T, int64_t m, int64_t n,
+                                             int32_t r);
+int grass_project_grad_batched(int32_t count, const void* const* dY, int64_t lddy,
+                               const void* const* X, int64_t ldx, int64_t T, int64_t m, int64_t n,
+                               const int32_t* const* idx, const float* const* rho, int32_t r,
+                               float* const* Gc, int64_t ldgc, void* ws, size_t ws_bytes,
+                               void* stream);
+int grass_adam_scatter_batched(int32_t count, const float* const* Gc, int64_t ldgc,
+                               float* const* M, float* const* V, float* const* U, int64_t ldstate,
+                               void* const* W, int wdt, int64_t m, int64_t n, int64_t ldw,
+                               const int32_t* const* idx, const float* const* rho, int32_t r,
+                               double lr, double beta1, double beta2, double eps, int32_t step,
+                               double alpha, void* stream);
+
+/*
  * Column form of the apply step, for layers projected on their input dimension
  * (Section 4.1: P acts on the smaller dimension of the gradient, so for m > n
  * the selection picks r of the n columns, G_C = G_W P, and W <- W + alpha U^T P^T):

@@ -275,3 +275,57 @@ def grass_profile_end():
     _check(load_library().grass_profile_end(kid, ms, ctypes.byref(n)), "grass_profile_end")
     timed = min(n.value, cap)
     return n.value, [(KERNEL_NAMES[kid[i]], float(ms[i])) for i in range(timed)]
+
+
+# ---- batched calls: `count` layers of one shape per launch ----
+_SIGNATURES_BATCHED = {
+    "grass_project_batched_workspace_bytes": (c_size_t, [c_int32, c_int64, c_int64, c_int64, c_int32]),
+    "grass_project_grad_batched": (c_int, [c_int32, c_void_p, c_int64, c_void_p, c_int64, c_int64,
+                                           c_int64, c_int64, c_void_p, c_void_p, c_int32, c_void_p,
+                                           c_int64, c_void_p, c_size_t, c_void_p]),
+    "grass_adam_scatter_batched": (c_int, [c_int32, c_void_p, c_int64, c_void_p, c_void_p, c_void_p,
+                                           c_int64, c_void_p, c_int, c_int64, c_int64, c_int64,
+                                           c_void_p, c_void_p, c_int32, c_double, c_double, c_double,
+                                           c_double, c_int32, c_double, c_void_p]),
+}
+_SIGNATURES.update(_SIGNATURES_BATCHED)
+
+
+def _ptr_array(tensors):
+    """Host array of device pointers (None entries become NULL); None -> NULL array."""
+    if tensors is None:
+        return None
+    arr = (c_void_p * len(tensors))(*[None if t is None else t.data_ptr() for t in tensors])
+    return arr
+
+
+def grass_project_batched_workspace_bytes(count: int, T: int, m: int, n: int, r: int) -> int:
+    return int(load_library().grass_project_batched_workspace_bytes(count, T, m, n, r))
+
+
+def grass_project_grad_batched(dYs, Xs, idxs, rhos, r, Gcs, ws) -> None:
+    count = len(dYs)
+    T, m = dYs[0].shape
+    n = Xs[0].shape[1]
+    for t in Gcs:
+        _require(t, torch.float32, "Gc")
+    for t in idxs:
+        _require(t, torch.int32, "idx")
+    keep = (_ptr_array(dYs), _ptr_array(Xs), _ptr_array(idxs), _ptr_array(rhos), _ptr_array(Gcs))
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(load_library().grass_project_grad_batched(
+        count, keep[0], _ld(dYs[0]), keep[1], _ld(Xs[0]), T, m, n, keep[2], keep[3], r, keep[4],
+        _ld(Gcs[0]), _ptr(ws), ws_bytes, _stream()), "grass_project_grad_batched")
+
+
+def grass_adam_scatter_batched(Gcs, Ms, Vs, Us, Ws, idxs, rhos, lr, beta1, beta2, eps, step,
+                               alpha) -> None:
+    count = len(Gcs)
+    r, n = Ms[0].shape
+    m = Ws[0].shape[0]
+    keep = (_ptr_array(Gcs), _ptr_array(Ms), _ptr_array(Vs), _ptr_array(Us), _ptr_array(Ws),
+            _ptr_array(idxs), _ptr_array(rhos))
+    _check(load_library().grass_adam_scatter_batched(
+        count, keep[0], _ld(Gcs[0]), keep[1], keep[2], keep[3], _ld(Ms[0]), keep[4],
+        _dtype_code(Ws[0]), m, n, _ld(Ws[0]), keep[5], keep[6], r, lr, beta1, beta2, eps, step,
+        alpha, _stream()), "grass_adam_scatter_batched")

@@ -20,13 +20,30 @@ namespace {
 
 constexpr int kThreads = 256;
 
+constexpr int kMaxGroup = 8;
+
+// Up to kMaxGroup same-shaped layers share one launch: blockIdx.z = layer of the group.
+struct UpdateGroup {
+  const float* Gc[kMaxGroup];
+  float* M[kMaxGroup];
+  float* V[kMaxGroup];
+  float* U[kMaxGroup];
+  void* W[kMaxGroup];
+  const int32_t* idx[kMaxGroup];
+  const float* rho[kMaxGroup];
+};
+
 template <typename T, bool VEC>
 __global__ void __launch_bounds__(kThreads)
-adam_scatter_kernel(const float* __restrict__ Gc, int64_t ldgc, float* __restrict__ M,
-                    float* __restrict__ V, float* __restrict__ U, int64_t ldstate,
-                    T* __restrict__ W, int64_t m, int64_t n, int64_t ldw,
-                    const int32_t* __restrict__ idx, const float* __restrict__ rho, int r,
-                    float alpha, AdamScalars a, int* status) {
+adam_scatter_kernel(const UpdateGroup grp, int64_t ldgc, int64_t ldstate, int64_t m, int64_t n,
+                    int64_t ldw, int r, float alpha, AdamScalars a, int* status) {
+  const float* __restrict__ Gc = grp.Gc[blockIdx.z];
+  float* __restrict__ M = grp.M[blockIdx.z];
+  float* __restrict__ V = grp.V[blockIdx.z];
+  float* __restrict__ U = grp.U[blockIdx.z];
+  T* __restrict__ W = static_cast<T*>(grp.W[blockIdx.z]);
+  const int32_t* __restrict__ idx = grp.idx[blockIdx.z];
+  const float* __restrict__ rho = grp.rho[blockIdx.z];
   const int j0 = blockIdx.y;
   const int row = idx[j0];
   if (j0 > 0 && idx[j0 - 1] == row) return;  // not the head of its run
@@ -89,29 +106,47 @@ adam_scatter_kernel(const float* __restrict__ Gc, int64_t ldgc, float* __restric
 }
 
 template <typename T>
-int launch(const float* Gc, int64_t ldgc, float* M, float* V, float* U, int64_t ldstate, void* W,
-           int64_t m, int64_t n, int64_t ldw, const int32_t* idx, const float* rho, int r,
-           float alpha, const AdamScalars& a, cudaStream_t s) {
+int launch(int count, const UpdateGroup& grp, int64_t ldgc, int64_t ldstate, int64_t m, int64_t n,
+           int64_t ldw, int r, float alpha, const AdamScalars& a, cudaStream_t s) {
   constexpr int N = WTraits<T>::N;
   cudaError_t err;
   int* status = status_word(&err);
   if (status == nullptr) GRASS_CUDA_TRY(err);
-  const bool vec = (n % N == 0) && (ldw % N == 0) && (ldgc % 4 == 0) && (ldstate % 4 == 0) &&
-                   aligned_to(W, 16) && aligned_to(Gc, 16) && aligned_to(M, 16) &&
-                   aligned_to(V, 16) && (U == nullptr || aligned_to(U, 16));
+  bool vec = (n % N == 0) && (ldw % N == 0) && (ldgc % 4 == 0) && (ldstate % 4 == 0);
+  for (int g = 0; g < count; ++g)
+    vec = vec && aligned_to(grp.W[g], 16) && aligned_to(grp.Gc[g], 16) && aligned_to(grp.M[g], 16) &&
+          aligned_to(grp.V[g], 16) && (grp.U[g] == nullptr || aligned_to(grp.U[g], 16));
   dim3 grid(static_cast<unsigned>((n + kThreads * N - 1) / (kThreads * N)),
-            static_cast<unsigned>(r));
+            static_cast<unsigned>(r), static_cast<unsigned>(count));
   ProfileScope prof(GRASS_K_ADAM_SCATTER, s);
   if (vec)
-    adam_scatter_kernel<T, true><<<grid, kThreads, 0, s>>>(Gc, ldgc, M, V, U, ldstate,
-                                                           static_cast<T*>(W), m, n, ldw, idx, rho,
-                                                           r, alpha, a, status);
+    adam_scatter_kernel<T, true><<<grid, kThreads, 0, s>>>(grp, ldgc, ldstate, m, n, ldw, r, alpha,
+                                                           a, status);
   else
-    adam_scatter_kernel<T, false><<<grid, kThreads, 0, s>>>(Gc, ldgc, M, V, U, ldstate,
-                                                            static_cast<T*>(W), m, n, ldw, idx, rho,
-                                                            r, alpha, a, status);
+    adam_scatter_kernel<T, false><<<grid, kThreads, 0, s>>>(grp, ldgc, ldstate, m, n, ldw, r, alpha,
+                                                            a, status);
   GRASS_LAUNCH_CHECK();
   return GRASS_OK;
+}
+
+int run(int count, const UpdateGroup& grp, int wdt, int64_t ldgc, int64_t ldstate, int64_t m,
+        int64_t n, int64_t ldw, int r, double lr, double beta1, double beta2, double eps, int step,
+        double alpha, cudaStream_t s) {
+  if (m < 1 || n < 1 || r < 1 || r > 65535 || ldgc < n || ldstate < n || ldw < n ||
+      m > 0x7fffffffLL)
+    return GRASS_ERR_INVALID_ARG;
+  for (int g = 0; g < count; ++g)
+    if (grp.Gc[g] == nullptr || grp.M[g] == nullptr || grp.V[g] == nullptr ||
+        grp.W[g] == nullptr || grp.idx[g] == nullptr)
+      return GRASS_ERR_INVALID_ARG;
+  if (!adam_args_ok(lr, beta1, beta2, eps, step)) return GRASS_ERR_INVALID_ARG;
+  const AdamScalars a = make_adam_scalars(lr, beta1, beta2, eps, step);
+  const float al = static_cast<float>(alpha);
+  if (wdt == GRASS_F32)
+    return launch<float>(count, grp, ldgc, ldstate, m, n, ldw, r, al, a, s);
+  if (wdt == GRASS_BF16)
+    return launch<__nv_bfloat16>(count, grp, ldgc, ldstate, m, n, ldw, r, al, a, s);
+  return GRASS_ERR_UNSUPPORTED;
 }
 
 }  // namespace
@@ -122,17 +157,33 @@ extern "C" int grass_adam_scatter(const float* Gc, int64_t ldgc, float* M, float
                                   int64_t ldw, const int32_t* idx, const float* rho, int32_t r,
                                   double lr, double beta1, double beta2, double eps, int32_t step,
                                   double alpha, void* stream) {
-  using namespace grass;
-  if (Gc == nullptr || M == nullptr || V == nullptr || W == nullptr || idx == nullptr || m < 1 ||
-      n < 1 || r < 1 || r > 65535 || ldgc < n || ldstate < n || ldw < n || m > 0x7fffffffLL)
+  grass::UpdateGroup grp;
+  for (int g = 0; g < grass::kMaxGroup; ++g) {
+    grp.Gc[g] = Gc; grp.M[g] = M; grp.V[g] = V; grp.U[g] = U; grp.W[g] = W;
+    grp.idx[g] = idx; grp.rho[g] = rho;
+  }
+  return grass::run(1, grp, wdt, ldgc, ldstate, m, n, ldw, r, lr, beta1, beta2, eps, step, alpha,
+                    static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int grass_adam_scatter_batched(int32_t count, const float* const* Gc, int64_t ldgc,
+                                          float* const* M, float* const* V, float* const* U,
+                                          int64_t ldstate, void* const* W, int wdt, int64_t m,
+                                          int64_t n, int64_t ldw, const int32_t* const* idx,
+                                          const float* const* rho, int32_t r, double lr,
+                                          double beta1, double beta2, double eps, int32_t step,
+                                          double alpha, void* stream) {
+  if (count < 1 || count > grass::kMaxGroup || Gc == nullptr || M == nullptr || V == nullptr ||
+      W == nullptr || idx == nullptr)
     return GRASS_ERR_INVALID_ARG;
-  if (!adam_args_ok(lr, beta1, beta2, eps, step)) return GRASS_ERR_INVALID_ARG;
-  const AdamScalars a = make_adam_scalars(lr, beta1, beta2, eps, step);
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const float al = static_cast<float>(alpha);
-  if (wdt == GRASS_F32)
-    return launch<float>(Gc, ldgc, M, V, U, ldstate, W, m, n, ldw, idx, rho, r, al, a, s);
-  if (wdt == GRASS_BF16)
-    return launch<__nv_bfloat16>(Gc, ldgc, M, V, U, ldstate, W, m, n, ldw, idx, rho, r, al, a, s);
-  return GRASS_ERR_UNSUPPORTED;
+  grass::UpdateGroup grp;
+  for (int g = 0; g < grass::kMaxGroup; ++g) {
+    const int gi = g < count ? g : 0;
+    grp.Gc[g] = Gc[gi]; grp.M[g] = M[gi]; grp.V[g] = V[gi];
+    grp.U[g] = U != nullptr ? U[gi] : nullptr;
+    grp.W[g] = W[gi]; grp.idx[g] = idx[gi];
+    grp.rho[g] = rho != nullptr ? rho[gi] : nullptr;
+  }
+  return grass::run(count, grp, wdt, ldgc, ldstate, m, n, ldw, r, lr, beta1, beta2, eps, step, alpha,
+                    static_cast<cudaStream_t>(stream));
 }

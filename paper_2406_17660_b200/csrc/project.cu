@@ -30,7 +30,7 @@ struct TcPlan {
 // n-tiles (MB) make more, smaller CTAs, which cuts partial traffic when the
 // output is tiny; larger ones cut the number of times the gathered operand is
 // re-read.  The result depends only on (T, n, r), so it is reproducible.
-TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false) {
+TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false, int groups = 1) {
   TcPlan p;
   const int r64 = static_cast<int>(round_up(static_cast<size_t>(r), 64));
   p.r_blocks = (r64 + 511) / 512;
@@ -53,7 +53,8 @@ TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false) {
       if (pair && n <= static_cast<int64_t>(mb) * 128) continue;  // nothing for the second CTA
       const int cta_cols = mb * 128 * (pair ? 2 : 1);
       const int n_tiles = static_cast<int>((n + cta_cols - 1) / cta_cols);
-      const int64_t tiles = static_cast<int64_t>(n_tiles) * p.r_blocks * (pair ? 2 : 1);  // CTAs
+      const int64_t tiles =
+          static_cast<int64_t>(n_tiles) * p.r_blocks * (pair ? 2 : 1) * groups;  // CTAs per split
       // clocks per 32-token block: tensor time, or (single CTA) the shared-memory ceiling
       double clk_per_block = static_cast<double>(mb) * p.r_cta;
       if (!pair) clk_per_block *= 1.4;
@@ -65,7 +66,7 @@ TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false) {
         const int64_t waves = (ctas + kSmCount - 1) / kSmCount;
         const double blocks_per_cta = static_cast<double>((p.k_blocks + s - 1) / s);
         double cost = waves * (blocks_per_cta * clk_per_block + fixed);
-        if (s > 1) cost += 8.0 * s * static_cast<double>(r) * n / hbm_bytes_per_clk;
+        if (s > 1) cost += 8.0 * s * groups * static_cast<double>(r) * n / hbm_bytes_per_clk;
         if (cost < best) {
           best = cost;
           p.MB = mb;
@@ -124,8 +125,7 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
 }
 
 template <int MB, int NSLAB, bool PAIR>
-int launch_tc_one(dim3 grid, size_t smem, cudaStream_t s, const CUtensorMap& tmX,
-                  const CUtensorMap& tmA, const TcParams& p) {
+int launch_tc_one(dim3 grid, size_t smem, cudaStream_t s, const TcMaps& maps, const TcParams& p) {
   static bool attr_set[64] = {false};
   int dev = 0;
   GRASS_CUDA_TRY(cudaGetDevice(&dev));
@@ -149,19 +149,19 @@ int launch_tc_one(dim3 grid, size_t smem, cudaStream_t s, const CUtensorMap& tmX
   cfg.numAttrs = 1;
   {
     ProfileScope prof(GRASS_K_PROJECT_TC, s);
-    GRASS_CUDA_TRY(cudaLaunchKernelEx(&cfg, project_tc_kernel<MB, NSLAB, PAIR>, tmX, tmA, p));
+    GRASS_CUDA_TRY(cudaLaunchKernelEx(&cfg, project_tc_kernel<MB, NSLAB, PAIR>, maps, p));
   }
   return GRASS_OK;
 }
 
 // (MB, NSLAB) with MB * 64 * NSLAB <= 512 TMEM columns; pairs need an even NSLAB.
 int launch_tc(int MB, int nslab, bool pair, dim3 grid, size_t smem, cudaStream_t s,
-              const CUtensorMap& tmX, const CUtensorMap& tmA, const TcParams& p) {
+              const TcMaps& maps, const TcParams& p) {
 #define GRASS_TC_CASE(mb, ns)                                                                  \
   if (MB == mb && nslab == ns && !pair)                                                        \
-    return launch_tc_one<mb, ns, false>(grid, smem, s, tmX, tmA, p)
+    return launch_tc_one<mb, ns, false>(grid, smem, s, maps, p)
 #define GRASS_TC_PAIR(mb, ns)                                                                  \
-  if (MB == mb && nslab == ns && pair) return launch_tc_one<mb, ns, true>(grid, smem, s, tmX, tmA, p)
+  if (MB == mb && nslab == ns && pair) return launch_tc_one<mb, ns, true>(grid, smem, s, maps, p)
   GRASS_TC_CASE(1, 1); GRASS_TC_CASE(1, 2); GRASS_TC_CASE(1, 3); GRASS_TC_CASE(1, 4);
   GRASS_TC_CASE(1, 5); GRASS_TC_CASE(1, 6); GRASS_TC_CASE(1, 7); GRASS_TC_CASE(1, 8);
   GRASS_TC_CASE(2, 1); GRASS_TC_CASE(2, 2); GRASS_TC_CASE(2, 3); GRASS_TC_CASE(2, 4);
@@ -178,8 +178,6 @@ size_t norm_part_bytes(int64_t m, int64_t n) {
                       sizeof(float), 256);
 }
 
-// norms != NULL: row-norm mode (idx NULL, r == m): the GEMM's epilogue reduces squares instead
-// of storing the gradient, then norms_finalize_kernel adds the per-column-group partials.
 // fp32 path: split the tokens when the output has too few 64 x 64 tiles to occupy the GPU.
 struct Fp32Plan {
   int split;
@@ -217,42 +215,67 @@ TcPlan make_norms_plan(int64_t T, int64_t n, int r) {
   return make_plan(T, n, r, false);
 }
 
-int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T, int64_t m,
-                 int64_t n, const int32_t* idx, const float* rho, int r, float* Gc, int64_t ldgc,
-                 float* norms, void* ws, size_t ws_bytes, cudaStream_t s) {
-  if (!aligned_to(X, 16) || ldx % 8 != 0) return GRASS_ERR_ALIGNMENT;
-  if (idx == nullptr && (!aligned_to(dY, 16) || lddy % 8 != 0)) return GRASS_ERR_ALIGNMENT;
-  const TcPlan plan = norms != nullptr ? make_norms_plan(T, n, r) : make_plan(T, n, r);
-  const bool gather = idx != nullptr;
+// Projection of `count` same-shaped layers in one set of launches (count = 1 for the plain
+// call).  norms != NULL (count must be 1): row-norm mode (idx NULL, r == m): the GEMM's epilogue
+// reduces squares instead of storing the gradient, then the partial sums are finalised.
+// Workspace layout: per layer [gathered operand][split-K partials], layers back to back.
+int project_bf16(int count, const void* const* dY, int64_t lddy, const void* const* X, int64_t ldx,
+                 int64_t T, int64_t m, int64_t n, const int32_t* const* idx,
+                 const float* const* rho, int r, float* const* Gc, int64_t ldgc, float* norms,
+                 void* ws, size_t ws_bytes, cudaStream_t s) {
+  if (count < 1 || count > kTcMaxGroup || (norms != nullptr && count != 1))
+    return GRASS_ERR_INVALID_ARG;
+  const bool gather = idx != nullptr && idx[0] != nullptr;
+  for (int g = 0; g < count; ++g) {
+    if (dY[g] == nullptr || X[g] == nullptr || (norms == nullptr && Gc[g] == nullptr))
+      return GRASS_ERR_INVALID_ARG;
+    if (gather != (idx != nullptr && idx[g] != nullptr)) return GRASS_ERR_INVALID_ARG;
+    if (!aligned_to(X[g], 16) || ldx % 8 != 0) return GRASS_ERR_ALIGNMENT;
+    if (!gather && (!aligned_to(dY[g], 16) || lddy % 8 != 0)) return GRASS_ERR_ALIGNMENT;
+  }
+  const TcPlan plan = norms != nullptr ? make_norms_plan(T, n, r) : make_plan(T, n, r, false, count);
   const bool fused_norms = norms != nullptr && plan.split_k == 1;
-  const size_t need = fused_norms ? norm_part_bytes(m, n)
-                                  : (gather ? plan.ag_bytes : 0) + plan.part_bytes;
+  const size_t per_layer = fused_norms ? norm_part_bytes(m, n)
+                                       : (gather ? plan.ag_bytes : 0) + plan.part_bytes;
+  const size_t need = per_layer * count;
   if (need > 0 && (ws == nullptr || !aligned_to(ws, 256) || ws_bytes < need))
     return GRASS_ERR_WORKSPACE;
   cudaError_t err;
   int* status = status_word(&err);
   if (status == nullptr) GRASS_CUDA_TRY(err);
 
-  char* wsp = static_cast<char*>(ws);
-  CUtensorMap tmX, tmA;
-  if (!make_map(&tmX, X, T, n, ldx, plan.bk)) return GRASS_ERR_CUDA;
-  if (gather) {
-    __nv_bfloat16* Ag = reinterpret_cast<__nv_bfloat16*>(wsp);
-    const __nv_bfloat16* dYb = static_cast<const __nv_bfloat16*>(dY);
-    {
-      ProfileScope prof(GRASS_K_GATHER, s);
-      const int ni = plan.r_pad >= 256 ? 8 : plan.r_pad / 32;   // r_pad is a multiple of 64
-      dim3 ggrid(static_cast<unsigned>((plan.r_pad + 32 * ni - 1) / (32 * ni)),
-                 static_cast<unsigned>((T + kGatherTokens - 1) / kGatherTokens));
-      gather_cols_kernel<<<ggrid, kGatherThreads, 0, s>>>(dYb, lddy, static_cast<int>(T),
-                                                          static_cast<int>(m), idx, r, plan.r_pad,
-                                                          ni, Ag, status);
+  TcMaps maps;
+  GatherGroup gg;
+  float* part[kTcMaxGroup];
+  for (int g = 0; g < count; ++g) {
+    char* wsp = static_cast<char*>(ws) + per_layer * g;
+    if (!make_map(&maps.x[g], X[g], T, n, ldx, plan.bk)) return GRASS_ERR_CUDA;
+    if (gather) {
+      gg.dY[g] = static_cast<const __nv_bfloat16*>(dY[g]);
+      gg.idx[g] = idx[g];
+      gg.Ag[g] = reinterpret_cast<__nv_bfloat16*>(wsp);
+      if (!make_map(&maps.a[g], gg.Ag[g], T, plan.r_pad, plan.r_pad, plan.bk)) return GRASS_ERR_CUDA;
+      wsp += plan.ag_bytes;
+    } else {
+      if (!make_map(&maps.a[g], dY[g], T, m, lddy, plan.bk)) return GRASS_ERR_CUDA;
     }
+    part[g] = reinterpret_cast<float*>(wsp);
+  }
+  for (int g = count; g < kTcMaxGroup; ++g) {
+    maps.x[g] = maps.x[0];
+    maps.a[g] = maps.a[0];
+    gg.dY[g] = nullptr; gg.idx[g] = nullptr; gg.Ag[g] = nullptr;
+  }
+  if (gather) {
+    ProfileScope prof(GRASS_K_GATHER, s);
+    const int ni = plan.r_pad >= 256 ? 8 : plan.r_pad / 32;   // r_pad is a multiple of 64
+    dim3 ggrid(static_cast<unsigned>((plan.r_pad + 32 * ni - 1) / (32 * ni)),
+               static_cast<unsigned>((T + kGatherTokens - 1) / kGatherTokens),
+               static_cast<unsigned>(count));
+    gather_cols_kernel<<<ggrid, kGatherThreads, 0, s>>>(gg, lddy, static_cast<int>(T),
+                                                        static_cast<int>(m), r, plan.r_pad, ni,
+                                                        status);
     GRASS_LAUNCH_CHECK();
-    if (!make_map(&tmA, Ag, T, plan.r_pad, plan.r_pad, plan.bk)) return GRASS_ERR_CUDA;
-    wsp += plan.ag_bytes;
-  } else {
-    if (!make_map(&tmA, dY, T, m, lddy, plan.bk)) return GRASS_ERR_CUDA;
   }
 
   TcParams p;
@@ -262,27 +285,28 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
   p.k_blocks = plan.k_blocks;
   p.split_k = plan.split_k;
   p.status = status;
-  p.norm_part = fused_norms ? reinterpret_cast<float*>(wsp) : nullptr;
+  p.norm_part = fused_norms ? part[0] : nullptr;
   p.ld_norm = static_cast<long long>(round_up(static_cast<size_t>(m), 32));
   if (getenv("GRASS_DEBUG_PLAN") != nullptr)
-    fprintf(stderr, "grass plan T=%lld n=%lld r=%d: r_cta=%d r_blocks=%d MB=%d n_blocks=%d "
-                    "split_k=%d stages=%d pair=%d\n", static_cast<long long>(T), static_cast<long long>(n),
-            r, plan.r_cta, plan.r_blocks, plan.MB, plan.n_blocks, plan.split_k, plan.stages,
-            plan.pair ? 1 : 0);
-  if (plan.split_k == 1) {
-    p.out = Gc;            // unused in row-norm mode
-    p.ld_out = ldgc;
-    p.split_stride = 0;
-    p.rho = rho;
-  } else {
-    p.out = reinterpret_cast<float*>(wsp);
-    p.ld_out = plan.ld_part;
-    p.split_stride = static_cast<long long>(r) * plan.ld_part;
-    p.rho = nullptr;
+    fprintf(stderr, "grass plan T=%lld n=%lld r=%d x%d: r_cta=%d r_blocks=%d MB=%d n_blocks=%d "
+                    "split_k=%d stages=%d pair=%d\n", static_cast<long long>(T),
+            static_cast<long long>(n), r, count, plan.r_cta, plan.r_blocks, plan.MB, plan.n_blocks,
+            plan.split_k, plan.stages, plan.pair ? 1 : 0);
+  for (int g = 0; g < kTcMaxGroup; ++g) {
+    const int gi = g < count ? g : 0;
+    if (plan.split_k == 1) {
+      p.out[g] = Gc != nullptr ? Gc[gi] : nullptr;   // unused in row-norm mode
+      p.rho[g] = rho != nullptr ? rho[gi] : nullptr;
+    } else {
+      p.out[g] = part[gi];
+      p.rho[g] = nullptr;
+    }
   }
+  p.ld_out = plan.split_k == 1 ? ldgc : plan.ld_part;
+  p.split_stride = plan.split_k == 1 ? 0 : static_cast<long long>(r) * plan.ld_part;
   dim3 grid(static_cast<unsigned>(plan.n_blocks), static_cast<unsigned>(plan.r_blocks),
-            static_cast<unsigned>(plan.split_k));
-  const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, grid, plan.smem_bytes, s, tmX, tmA, p);
+            static_cast<unsigned>(plan.split_k * count));
+  const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, grid, plan.smem_bytes, s, maps, p);
   if (rc != GRASS_OK) return rc;
   if (norms != nullptr) {
     ProfileScope prof(GRASS_K_ROW_NORMS, s);
@@ -291,20 +315,28 @@ int project_bf16(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64
           p.norm_part, p.ld_norm, static_cast<int>((n + 31) / 32), static_cast<int>(m), norms);
     else
       splitk_rownorms_kernel<<<static_cast<unsigned>(m), 256, 0, s>>>(
-          p.out, plan.ld_part, p.split_stride, plan.split_k, static_cast<int>(m),
+          part[0], plan.ld_part, p.split_stride, plan.split_k, static_cast<int>(m),
           static_cast<int>(n), norms);
     GRASS_LAUNCH_CHECK();
     return GRASS_OK;
   }
   if (plan.split_k > 1) {
-    const int vec = (n % 4 == 0) && (ldgc % 4 == 0) && aligned_to(Gc, 16);
+    ReduceGroup rg;
+    int vec = (n % 4 == 0) && (ldgc % 4 == 0);
+    for (int g = 0; g < kTcMaxGroup; ++g) {
+      const int gi = g < count ? g : 0;
+      rg.part[g] = part[gi];
+      rg.rho[g] = rho != nullptr ? rho[gi] : nullptr;
+      rg.Gc[g] = Gc[gi];
+      vec = vec && aligned_to(Gc[gi], 16);
+    }
     const long long work = static_cast<long long>(r) * (vec ? n / 4 : n);
     long long blocks = (work + 255) / 256;
     if (blocks > kSmCount * 32) blocks = kSmCount * 32;
     ProfileScope prof(GRASS_K_SPLITK_REDUCE, s);
-    splitk_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(
-        p.out, plan.ld_part, p.split_stride, plan.split_k, r, static_cast<int>(n), rho, Gc, ldgc,
-        vec);
+    splitk_reduce_kernel<<<dim3(static_cast<unsigned>(blocks), static_cast<unsigned>(count)), 256, 0,
+                           s>>>(rg, plan.ld_part, p.split_stride, plan.split_k, r,
+                                static_cast<int>(n), ldgc, vec);
     GRASS_LAUNCH_CHECK();
   }
   return GRASS_OK;
@@ -335,7 +367,8 @@ extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, i
   if (r > m) return GRASS_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dt == GRASS_BF16)
-    return project_bf16(dY, lddy, X, ldx, T, m, n, idx, rho, r, Gc, ldgc, nullptr, ws, ws_bytes, s);
+    return project_bf16(1, &dY, lddy, &X, ldx, T, m, n, idx != nullptr ? &idx : nullptr, &rho, r,
+                        &Gc, ldgc, nullptr, ws, ws_bytes, s);
   if (dt != GRASS_F32) return GRASS_ERR_UNSUPPORTED;
   cudaError_t err;
   int* status = status_word(&err);
@@ -360,12 +393,38 @@ extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, i
     long long blocks = (work + 255) / 256;
     if (blocks > kSmCount * 32) blocks = kSmCount * 32;
     ProfileScope prof(GRASS_K_SPLITK_REDUCE, s);
+    ReduceGroup rg;
+    for (int g = 0; g < kTcMaxGroup; ++g) { rg.part[g] = out; rg.rho[g] = rho; rg.Gc[g] = Gc; }
     splitk_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(
-        out, fp.ld_part, static_cast<long long>(r) * fp.ld_part, fp.split, r, static_cast<int>(n),
-        rho, Gc, ldgc, vec);
+        rg, fp.ld_part, static_cast<long long>(r) * fp.ld_part, fp.split, r, static_cast<int>(n),
+        ldgc, vec);
     GRASS_LAUNCH_CHECK();
   }
   return GRASS_OK;
+}
+
+extern "C" size_t grass_project_batched_workspace_bytes(int32_t count, int64_t T, int64_t m,
+                                                        int64_t n, int32_t r) {
+  (void)m;
+  if (count < 1 || count > grass::kTcMaxGroup || T < 1 || n < 1 || r < 1) return 0;
+  const grass::TcPlan plan = grass::make_plan(T, n, r, false, count);
+  return (plan.ag_bytes + plan.part_bytes) * static_cast<size_t>(count) + 256;
+}
+
+extern "C" int grass_project_grad_batched(int32_t count, const void* const* dY, int64_t lddy,
+                                          const void* const* X, int64_t ldx, int64_t T, int64_t m,
+                                          int64_t n, const int32_t* const* idx,
+                                          const float* const* rho, int32_t r, float* const* Gc,
+                                          int64_t ldgc, void* ws, size_t ws_bytes, void* stream) {
+  using namespace grass;
+  if (count < 1 || count > kTcMaxGroup || dY == nullptr || X == nullptr || idx == nullptr ||
+      Gc == nullptr || T < 1 || m < 1 || n < 1 || r < 1 || r > m || lddy < m || ldx < n ||
+      ldgc < n || T > 0x7fffffffLL || m > 0x7fffffffLL || n > 0x7fffffffLL)
+    return GRASS_ERR_INVALID_ARG;
+  for (int g = 0; g < count; ++g)
+    if (idx[g] == nullptr) return GRASS_ERR_INVALID_ARG;
+  return project_bf16(count, dY, lddy, X, ldx, T, m, n, idx, rho, r, Gc, ldgc, nullptr, ws, ws_bytes,
+                      static_cast<cudaStream_t>(stream));
 }
 
 extern "C" size_t grass_grad_row_norms_workspace_bytes(int64_t T, int64_t m, int64_t n, int dt) {
@@ -387,8 +446,8 @@ extern "C" int grass_grad_row_norms(const void* dY, int64_t lddy, const void* X,
     return GRASS_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dt == GRASS_BF16)
-    return project_bf16(dY, lddy, X, ldx, T, m, n, nullptr, nullptr, static_cast<int>(m), nullptr,
-                        0, norms, ws, ws_bytes, s);
+    return project_bf16(1, &dY, lddy, &X, ldx, T, m, n, nullptr, nullptr, static_cast<int>(m),
+                        nullptr, 0, norms, ws, ws_bytes, s);
   if (dt != GRASS_F32) return GRASS_ERR_UNSUPPORTED;
   // fp32 path: the (small) gradient is formed in the workspace and reduced by grass_row_norms
   if (ws == nullptr || !aligned_to(ws, 256) ||

@@ -67,14 +67,23 @@ __host__ __device__ constexpr int tc_stages(int MB, int A_SLABS) {
              : (kTcSmemBudget - 1024) / tc_stage_bytes(MB, A_SLABS);
 }
 
+constexpr int kTcMaxGroup = 8;
+
+// The X and gathered-dY tensor maps of every layer of the group (kernel parameter space).
+struct TcMaps {
+  CUtensorMap x[kTcMaxGroup];
+  CUtensorMap a[kTcMaxGroup];
+};
+
 struct TcParams {
   int T, n, r;          // logical sizes
   int k_blocks;         // ceil(T / tokens per stage)
   int split_k;          // gridDim.z
-  float* out;           // split_k == 1: Gc, else partials [split][r][ld_out]
+  // Up to kTcMaxGroup same-shaped layers share one launch: blockIdx.z = group * split_k + split.
+  float* out[kTcMaxGroup];        // split_k == 1: Gc, else partials [split][r][ld_out]
   long long ld_out;     // row pitch of out, elements
   long long split_stride;  // elements between partials of consecutive splits
-  const float* rho;     // applied here only when split_k == 1 (may be NULL)
+  const float* rho[kTcMaxGroup];  // applied here only when split_k == 1 (entries may be NULL)
   float* norm_part;     // non-NULL: row-norm mode.  Nothing of D is stored; instead
                         // norm_part[g * ld_norm + j] = sum of D[j, c]^2 over the 32 columns c of group g
   long long ld_norm;
@@ -99,8 +108,7 @@ __device__ __forceinline__ float warp_transpose_sum(float (&x)[32], int lane) {
 
 template <int MB, int NSLAB, bool PAIR>
 __global__ void __launch_bounds__(kTcThreads, 1)
-project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA,
-                  const TcParams p) {
+project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   constexpr int R_CTA = 64 * NSLAB;          // selected rows per CTA tile (per pair if PAIR)
   constexpr int X_SLABS = 2 * MB;
   constexpr int A_SLABS = PAIR ? NSLAB / 2 : NSLAB;   // slabs of the gathered operand this CTA stages
@@ -132,7 +140,10 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   const int r0 = blockIdx.y * R_CTA;
   // this CTA's token blocks: [kb_begin, kb_begin + kb_count)
   const int kb_per = p.k_blocks / p.split_k, kb_rem = p.k_blocks % p.split_k;
-  const int z = blockIdx.z;
+  const int grp = blockIdx.z / p.split_k;          // which layer of the group
+  const int z = blockIdx.z - grp * p.split_k;      // which token slice
+  const CUtensorMap* tmX = &maps.x[grp];
+  const CUtensorMap* tmA = &maps.a[grp];
   const int kb_begin = z * kb_per + (z < kb_rem ? z : kb_rem);
   const int kb_count = kb_per + (z < kb_rem ? 1 : 0);
 
@@ -145,8 +156,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     }
     ptx::mbar_init(&bar_accum, 1);
     ptx::fence_mbar_init();
-    ptx::prefetch_tensormap(&tmX);
-    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(tmX);
+    ptx::prefetch_tensormap(tmA);
   }
   if (warp == 1) {
     if (PAIR) {
@@ -166,7 +177,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   if (warp == 0) {
     // ================= TMA producer: one lane per slab =================
     const bool is_x = lane < X_SLABS;
-    const CUtensorMap* map = is_x ? &tmX : &tmA;
+    const CUtensorMap* map = is_x ? tmX : tmA;
     int xcoord;
     if (is_x) {
       xcoord = c_base + (lane >> 1) * C_STEP + (lane & 1) * 64;
@@ -278,8 +289,9 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     }
     if (ok && *abort_flag == 0) {
       ptx::fence_tc_after_sync();
-      float* out = p.out + static_cast<long long>(z) * p.split_stride;
-      const bool scale = p.split_k == 1 && p.rho != nullptr;
+      float* out = p.out[grp] + static_cast<long long>(z) * p.split_stride;
+      const float* rho = p.rho[grp];
+      const bool scale = p.split_k == 1 && rho != nullptr;
       const long long ld = p.ld_out;
 #pragma unroll 1
       for (int chunk = half; chunk < MB * (R_CTA / 32); chunk += 2) {
@@ -303,7 +315,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           continue;
         }
         float my_rho = 1.f;
-        if (scale && row0 + lane < p.r) my_rho = __ldg(p.rho + row0 + lane);
+        if (scale && row0 + lane < p.r) my_rho = __ldg(rho + row0 + lane);
         float* dst = out + static_cast<long long>(row0) * ld + c;
         const int nvalid = p.r - row0 < 32 ? p.r - row0 : 32;
         if (nvalid == 32) {
@@ -339,15 +351,23 @@ project_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 // sector look-ups the load unit performs per useful byte.
 constexpr int kGatherThreads = 256;
 constexpr int kGatherTokens = 32;            // tokens per block
+struct GatherGroup {
+  const __nv_bfloat16* dY[kTcMaxGroup];
+  const int32_t* idx[kTcMaxGroup];
+  __nv_bfloat16* Ag[kTcMaxGroup];
+};
 
 // A warp owns one token at a time and 32 * ni consecutive j: lane l loads
 // j = jb + 32 i + l for i < ni, so one load instruction covers 32 neighbouring
 // selected columns (ascending idx: as few 32-byte sectors as the selection
 // allows) and one store instruction writes 64 contiguous bytes of Ag.
 __global__ void __launch_bounds__(kGatherThreads)
-gather_cols_kernel(const __nv_bfloat16* __restrict__ dY, long long lddy, int T, int m,
-                     const int32_t* __restrict__ idx, int r, int r_pad, int ni,
-                     __nv_bfloat16* __restrict__ Ag, int* status) {
+gather_cols_kernel(const GatherGroup grp, long long lddy, int T, int m, int r, int r_pad, int ni,
+                   int* status) {
+  // blockIdx.z = layer of the group
+  const __nv_bfloat16* __restrict__ dY = grp.dY[blockIdx.z];
+  const int32_t* __restrict__ idx = grp.idx[blockIdx.z];
+  __nv_bfloat16* __restrict__ Ag = grp.Ag[blockIdx.z];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int jb = blockIdx.x * (32 * ni);
   int rows[8];
@@ -381,11 +401,20 @@ gather_cols_kernel(const __nv_bfloat16* __restrict__ dY, long long lddy, int T, 
   }
 }
 
+struct ReduceGroup {
+  const float* part[kTcMaxGroup];
+  const float* rho[kTcMaxGroup];
+  float* Gc[kTcMaxGroup];
+};
+
 // Gc[j, c] = rho_j * sum_s part[s][j][c], splits added in increasing s.
 __global__ void __launch_bounds__(256)
-splitk_reduce_kernel(const float* __restrict__ part, long long ld_part, long long split_stride,
-                     int split_k, int r, int n, const float* __restrict__ rho,
-                     float* __restrict__ Gc, long long ldgc, int vec) {
+splitk_reduce_kernel(const ReduceGroup grp, long long ld_part, long long split_stride, int split_k,
+                     int r, int n, long long ldgc, int vec) {
+  // blockIdx.y = layer of the group
+  const float* __restrict__ part = grp.part[blockIdx.y];
+  const float* __restrict__ rho = grp.rho[blockIdx.y];
+  float* __restrict__ Gc = grp.Gc[blockIdx.y];
   const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
   if (vec) {
     const int nv = n / 4;

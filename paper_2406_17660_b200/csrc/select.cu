@@ -104,7 +104,6 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
   extern __shared__ __align__(16) float s_dyn[];   // staged norms / scores, then hit counters
   __shared__ int s_hist[256];
   __shared__ int s_int[kWarps + 1];
-  __shared__ double s_dbl[kWarps + 1];
   __shared__ int s_flag;
   __shared__ uint32_t s_prefix;
   __shared__ int s_need;

@@ -101,3 +101,39 @@ class GrassLayer:
         else:
             B.grass_scatter_update(self.W, self.U, self.idx, self.rho, self.alpha)
         self.t += 1
+
+
+class GrassLayerGroup:
+    """Up to 8 layers of one shape (row selection, bf16) stepped together: their projections
+    run as one set of launches and so do their Adam + apply updates.  The layers keep their
+    own selection, state and weights; refresh iterations are done layer by layer."""
+
+    def __init__(self, layers, T, device="cuda"):
+        if not 1 <= len(layers) <= 8:
+            raise ValueError("a group holds 1 to 8 layers")
+        first = layers[0]
+        for l in layers:
+            if (l.W.shape, l.r, l.K, l.side) != (first.W.shape, first.r, first.K, "rows"):
+                raise ValueError("layers of a group must share shape, r, K and select rows")
+        self.layers = layers
+        nbytes = B.grass_project_batched_workspace_bytes(len(layers), T, first.m, first.n, first.r)
+        self.ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        self.stream = None
+
+    def step(self, dYs, Xs):
+        ls = self.layers
+        first = ls[0]
+        if first.t % first.K == 0:
+            for l, dY, X in zip(ls, dYs, Xs):
+                l.refresh(dY, X)
+        for l in ls:
+            l.adam_step += 1
+        B.grass_project_grad_batched(dYs, Xs, [l.idx for l in ls], [l.rho for l in ls], first.r,
+                                     [l.Gc for l in ls], self.ws)
+        B.grass_adam_scatter_batched([l.Gc for l in ls], [l.M for l in ls], [l.V for l in ls],
+                                     [l.U if l.keep_U else None for l in ls], [l.W for l in ls],
+                                     [l.idx for l in ls], [l.rho for l in ls], first.lr,
+                                     first.beta1, first.beta2, first.eps, first.adam_step,
+                                     first.alpha)
+        for l in ls:
+            l.t += 1
