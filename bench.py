@@ -229,7 +229,7 @@ def run_gpu(args):
     import paper_2406_17660_b200 as grass
     from paper_2406_17660_b200 import synthetic as syn
     from paper_2406_17660_b200 import workloads
-    from paper_2406_17660_b200.step import GrassLayer, GrassWorkspace
+    from paper_2406_17660_b200.step import GrassLayer, GrassLayerGroup, GrassWorkspace
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -272,13 +272,43 @@ def run_gpu(args):
         layers.append((pi, layer))
     in_bytes = sum(d.numel() * d.element_size() + x.numel() * x.element_size() for d, x in block_in)
 
+    # units of work: a single layer, or (--batched, bf16) a run of consecutive layers of one
+    # shape inside a block (q,k,v,o / gate,up / down) stepped by one set of launches.  A unit has
+    # one stream and one scratch; consecutive units alternate over the streams.
+    units = []
+    i = 0
+    while i < len(layers):
+        j = i + 1
+        if args.batched and wl.dtype == torch.bfloat16:
+            while (j < len(layers) and j - i < 8 and layers[j][1].W.shape == layers[i][1].W.shape
+                   and j // len(wl.shapes) == i // len(wl.shapes)):
+                j += 1
+        members = layers[i:j]
+        obj = members[0][1] if len(members) == 1 else GrassLayerGroup([l for _, l in members], wl.T,
+                                                                      device=dev)
+        units.append({"obj": obj, "pis": [pi for pi, _ in members], "layers": [l for _, l in members]})
+        i = j
+    for u, unit in enumerate(units):
+        unit["stream"] = streams[u % n_streams]
+        for l in unit["layers"]:
+            l.stream = unit["stream"]
+            l.ws = wss[u % n_streams]
+
+    def run_unit(unit, stream):
+        with torch.cuda.stream(stream):
+            if len(unit["layers"]) == 1:
+                unit["obj"].step(*block_in[unit["pis"][0]])
+            else:
+                unit["obj"].step([block_in[p][0] for p in unit["pis"]],
+                                 [block_in[p][1] for p in unit["pis"]])
+
+    single_stream = [False]
+
     def one_step():
         for st in streams[1:]:
             st.wait_stream(main_stream)
-        for pi, layer in layers:
-            dY, X = block_in[pi]
-            with torch.cuda.stream(layer.stream):
-                layer.step(dY, X)
+        for unit in units:
+            run_unit(unit, main_stream if single_stream[0] else unit["stream"])
         for st in streams[1:]:
             main_stream.wait_stream(st)
 
@@ -318,15 +348,12 @@ def run_gpu(args):
     cap = args.steps * len(layers) * 5 + n_refresh * len(layers) * 8 + 16
     # one stream for this pass: an event pair must bracket one kernel running alone, not a kernel
     # sharing the GPU with another layer's kernels
-    saved_streams = [layer.stream for _, layer in layers]
-    for _, layer in layers:
-        layer.stream = main_stream
+    single_stream[0] = True
     grass.grass_profile_begin(cap)
     for i in range(args.steps):
         one_step()
     launches, recs = grass.grass_profile_end()
-    for (_, layer), st in zip(layers, saved_streams):
-        layer.stream = st
+    single_stream[0] = False
     clocks = sampler.stop() if rank == 0 else None
     per_kernel = {}
     for name, ms in recs:
@@ -461,7 +488,7 @@ def run_gpu(args):
                        "inputs": "one block of distinct dY/X reused by every block",
                        "l2": f"inputs {in_bytes / 1e6:.0f} MB per step, larger than the 126 MB L2",
                        "parallelism": "replicas" if world > 1 else "single GPU",
-                       "streams": n_streams,
+                       "streams": n_streams, "batched": bool(args.batched),
                        "flops": "2rTn per layer-step + 2mTn per refresh"},
             "us_per_layer_step_regular": None if reg_ms is None else 1e3 * reg_ms / n_layers,
             "us_per_layer_step_refresh": None if ref_ms is None else 1e3 * ref_ms / n_layers,
@@ -489,6 +516,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--streams", type=int, default=2, help="streams that layers alternate over")
     ap.add_argument("--unfused", action="store_true", help="separate Adam and apply kernels")
+    ap.add_argument("--no-batched", dest="batched", action="store_false",
+                    help="one set of launches per layer instead of per run of same-shaped layers")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -119,6 +119,24 @@ class GrassLayerGroup:
         nbytes = B.grass_project_batched_workspace_bytes(len(layers), T, first.m, first.n, first.r)
         self.ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
         self.stream = None
+        # host arrays of device pointers: built once for the buffers the layers own, and once per
+        # distinct set of input tensors (the marshalling would otherwise dominate small layers)
+        pa = B._ptr_array
+        self._own = dict(idx=pa([l.idx for l in layers]), rho=pa([l.rho for l in layers]),
+                         Gc=pa([l.Gc for l in layers]), M=pa([l.M for l in layers]),
+                         V=pa([l.V for l in layers]), W=pa([l.W for l in layers]),
+                         U=pa([l.U if l.keep_U else None for l in layers]))
+        self._inputs = {}
+
+    def _input_arrays(self, dYs, Xs):
+        key = tuple(t.data_ptr() for t in dYs) + tuple(t.data_ptr() for t in Xs)
+        hit = self._inputs.get(key)
+        if hit is None:
+            if len(self._inputs) > 64:
+                self._inputs.clear()
+            hit = (B._ptr_array(dYs), B._ptr_array(Xs), B._ld(dYs[0]), B._ld(Xs[0]), dYs[0].shape[0])
+            self._inputs[key] = hit
+        return hit
 
     def step(self, dYs, Xs):
         ls = self.layers
@@ -128,12 +146,20 @@ class GrassLayerGroup:
                 l.refresh(dY, X)
         for l in ls:
             l.adam_step += 1
-        B.grass_project_grad_batched(dYs, Xs, [l.idx for l in ls], [l.rho for l in ls], first.r,
-                                     [l.Gc for l in ls], self.ws)
-        B.grass_adam_scatter_batched([l.Gc for l in ls], [l.M for l in ls], [l.V for l in ls],
-                                     [l.U if l.keep_U else None for l in ls], [l.W for l in ls],
-                                     [l.idx for l in ls], [l.rho for l in ls], first.lr,
-                                     first.beta1, first.beta2, first.eps, first.adam_step,
-                                     first.alpha)
-        for l in ls:
             l.t += 1
+        lib = B.load_library()
+        own = self._own
+        dYa, Xa, lddy, ldx, T = self._input_arrays(dYs, Xs)
+        stream = B._stream()
+        count, ld = len(ls), B._ld(first.Gc)
+        B._check(lib.grass_project_grad_batched(count, dYa, lddy, Xa, ldx, T, first.m, first.n,
+                                                own["idx"], own["rho"], first.r, own["Gc"], ld,
+                                                B._ptr(self.ws), self.ws.numel(), stream),
+                 "grass_project_grad_batched")
+        B._check(lib.grass_adam_scatter_batched(count, own["Gc"], ld, own["M"], own["V"], own["U"],
+                                                B._ld(first.M), own["W"], B._dtype_code(first.W),
+                                                first.W.shape[0], first.n, B._ld(first.W),
+                                                own["idx"], own["rho"], first.r, first.lr,
+                                                first.beta1, first.beta2, first.eps,
+                                                first.adam_step, first.alpha, stream),
+                 "grass_adam_scatter_batched")
