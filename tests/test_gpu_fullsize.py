@@ -75,3 +75,31 @@ def test_layer_step_on_sampled_rows(T, m, n, r, method):
         assert np.mean(Wn[k] != want) < 0.01
     untouched = np.setdiff1d(np.arange(m), idx)
     assert torch.equal(layer.W[untouched].cpu(), W[untouched])
+
+
+def test_batched_projection_at_7b_shape_on_sampled_rows():
+    """The q, k, v, o projections of a LLaMA-7B block stepped as one group, as bench.py does:
+    four layers of 4096 x 4096, T = 32768, r = 1024 in one set of launches."""
+    T, m, n, r, count = 32768, 4096, 4096, 1024, 4
+    dt = torch.bfloat16
+    rng = np.random.default_rng(99)
+    X = [syn.make_X(T, n, dt, seed0=21, proj=g) for g in range(count)]
+    dY = [syn.make_dY(T, m, dt, seed0=21, proj=g) for g in range(count)]
+    sig = [np.sort(rng.choice(m, r, replace=False)) for _ in range(count)]
+    rho = [(0.5 + rng.random(r)).astype(np.float32) for _ in range(count)]
+    Xd, dYd = [t.to(DEV) for t in X], [t.to(DEV) for t in dY]
+    idx = [torch.tensor(s, dtype=torch.int32, device=DEV) for s in sig]
+    rhod = [torch.tensor(x, device=DEV) for x in rho]
+    Gc = [torch.full((r, n), float("nan"), dtype=torch.float32, device=DEV) for _ in range(count)]
+    ws = torch.empty(grass.grass_project_batched_workspace_bytes(count, T, m, n, r),
+                     dtype=torch.uint8, device=DEV)
+    grass.grass_project_grad_batched(dYd, Xd, idx, rhod, r, Gc, ws)
+    grass.grass_device_status()
+    for g in range(count):
+        X64 = f64(X[g])
+        got = f64(Gc[g])
+        assert np.all(np.isfinite(got))
+        for j in rng.choice(r, 3, replace=False):
+            want = rho[g][j] * (X64.T @ f64(dY[g][:, sig[g][j]]))
+            err = np.linalg.norm(got[j] - want) / np.linalg.norm(want)
+            assert err <= 1e-2 and err <= 1e-4, (g, j, err)
