@@ -347,8 +347,8 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
 
 // Ag[t, j] = dY[t, idx[j]] (bf16 bits copied unchanged), zero for r <= j < r_pad.
 // HBM moves at least 32-byte sectors (16 bf16), so the copy reads 2 T m (1 - (1 - r/m)^16)
-// bytes of dY or more however it is written (practically all of dY from r/m = 1/16 up); what the kernel controls is how many
-// sector look-ups the load unit performs per useful byte.
+// bytes of dY or more however it is written (practically all of dY from r/m = 1/16 up);
+// what the kernel controls is how many sector look-ups the load unit performs per useful byte.
 constexpr int kGatherThreads = 256;
 constexpr int kGatherTokens = 32;            // tokens per block
 struct GatherGroup {
