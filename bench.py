@@ -29,11 +29,12 @@ if ROOT not in sys.path:
 METRIC = "TFLOP/s per layer-step (select+project+Adam+scatter)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised in profiles/project_tc_kernel_llama7b_q_r1024.md (None where no capture of
-# that workload exists).  The capture is of an n = 4096 launch (six of the seven projections of the
-# block); the n = 11008 launch scales with 2Tn + 2Tr to about 792 MB.
-NCU_TRAFFIC_BYTES = {"llama7b_block_r1024": 339.1e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel.  ncu captured
+# one n = 4096 layer (339.1 MB: X and the gathered operand each read once, see
+# profiles/project_tc_kernel_llama7b_q_r1024.md); traffic grows in proportion to the layers and
+# to 2Tn + 2Tr, so the three batched launches of a step move 4 x 339 MB (q,k,v,o), 2 x 339 MB
+# (gate, up) and about 792 MB (down): 942 MB per launch on average.  None where nothing was captured.
+NCU_TRAFFIC_BYTES = {"llama7b_block_r1024": 942e6}
 
 
 def load_peaks():
