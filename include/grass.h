@@ -206,7 +206,8 @@ int grass_subspace_adam(const float* Gc, int64_t ldgc, float* M, float* V, float
  *   idx  [r] ascending (as grass_select writes it); repeated rows must be
  *        adjacent: their terms are summed in fp32 in order of j and the row is
  *        written once (bf16: one round-to-nearest-even at the end).
- * A row index outside [0, m) is skipped and sets the status word.
+ * A row index outside [0, m) is skipped and sets the status word.  r <= 65535
+ * (one grid row per selected row).
  */
 int grass_scatter_update(void* W, int wdt, int64_t m, int64_t n, int64_t ldw, const float* U,
                          int64_t ldu, const int32_t* idx, const float* rho, int32_t r,

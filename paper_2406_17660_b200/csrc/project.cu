@@ -46,7 +46,8 @@ TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false, int gro
   p.MB = 1;
   p.split_k = 1;
   // GRASS_TC_NO_PAIR (diagnostic) keeps every CTA on its own MMA, for A/B timing
-  const bool can_pair = (p.r_cta % 128) == 0 && getenv("GRASS_TC_NO_PAIR") == nullptr;
+  static const bool no_pair = getenv("GRASS_TC_NO_PAIR") != nullptr;   // read once
+  const bool can_pair = (p.r_cta % 128) == 0 && !no_pair;
   p.pair = false;
   for (int mb = mb_max; mb >= 1; mb /= 2) {
     for (int pair = can_pair ? 1 : 0; pair >= 0; --pair) {
@@ -287,7 +288,8 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   p.status = status;
   p.norm_part = fused_norms ? part[0] : nullptr;
   p.ld_norm = static_cast<long long>(round_up(static_cast<size_t>(m), 32));
-  if (getenv("GRASS_DEBUG_PLAN") != nullptr)
+  static const bool debug_plan = getenv("GRASS_DEBUG_PLAN") != nullptr;   // read once
+  if (debug_plan)
     fprintf(stderr, "grass plan T=%lld n=%lld r=%d x%d: r_cta=%d r_blocks=%d MB=%d n_blocks=%d "
                     "split_k=%d stages=%d pair=%d\n", static_cast<long long>(T),
             static_cast<long long>(n), r, count, plan.r_cta, plan.r_blocks, plan.MB, plan.n_blocks,
