@@ -542,3 +542,36 @@ def test_batched_projection_and_update_match_the_oracle_layer_by_layer(count, T,
         assert torch.equal(M1, M[g]) and torch.equal(V1, V[g]) and torch.equal(W1, Wd[g])
         Mo, Vo, Uo = oracle.adam_update(np.zeros((r, n)), np.zeros((r, n)), want, 1e-3, 0.9, 0.999, 1e-8, 1)
         assert rel_fro(f64(M[g]), Mo) <= 1e-4
+
+
+# --------------------------------------------------------------------------- resume
+def test_resume_from_copied_state_is_bit_identical():
+    """All state is caller-owned buffers plus (t, adam_step); selection is a pure function of
+    (norms, seed, layer_id, epoch).  Six steps in one go equal three steps, a copy of the state
+    into a fresh layer, and three more."""
+    m, n, T, r, K = 512, 512, 1024, 128, 2
+    dt, method = torch.bfloat16, grass.SEL_MULTINOMIAL_NORM
+    W0 = syn.make_W(m, n, dt, seed0=31).to(DEV)
+    batches = [(syn.make_dY(T, m, dt, seed0=31, step=t).to(DEV), syn.make_X(T, n, dt, seed0=31, step=t).to(DEV))
+               for t in range(6)]
+
+    def fresh(W):
+        ws = grass.step.GrassWorkspace([(m, n)], T, r, dt, method)
+        return grass.GrassLayer(W, r, method, K, 0.25, 1e-3, reset_state=False, seed=77, layer_id=3,
+                                workspace=ws)
+
+    a = fresh(W0.clone())
+    for dY, X in batches:
+        a.step(dY, X)
+    b = fresh(W0.clone())
+    for dY, X in batches[:3]:
+        b.step(dY, X)
+    c = fresh(b.W.clone())
+    for name in ("M", "V", "idx", "rho"):
+        getattr(c, name).copy_(getattr(b, name))
+    c.t, c.adam_step = b.t, b.adam_step
+    for dY, X in batches[3:]:
+        c.step(dY, X)
+    grass.grass_device_status()
+    assert torch.equal(a.W, c.W) and torch.equal(a.M, c.M) and torch.equal(a.V, c.V)
+    assert torch.equal(a.idx, c.idx)
