@@ -227,6 +227,7 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   if (count < 1 || count > kTcMaxGroup || (norms != nullptr && count != 1))
     return GRASS_ERR_INVALID_ARG;
   const bool gather = idx != nullptr && idx[0] != nullptr;
+  if (gather && T > 65535LL * kGatherTokens) return GRASS_ERR_UNSUPPORTED;   // gather grid.y
   for (int g = 0; g < count; ++g) {
     if (dY[g] == nullptr || X[g] == nullptr || (norms == nullptr && Gc[g] == nullptr))
       return GRASS_ERR_INVALID_ARG;
