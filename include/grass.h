@@ -316,6 +316,10 @@ typedef enum {
 } grass_kernel_t;
 int grass_profile_begin(int32_t max_launches);
 int grass_profile_end(int32_t* kernel_id, float* ms, int32_t* n_launches);
+/* The same, plus start_ms[i] (host, may be NULL): when launch i began, in milliseconds after
+ * the first recorded launch began -- across streams, so overlap between streams is visible. */
+int grass_profile_end_timeline(int32_t* kernel_id, float* ms, float* start_ms,
+                               int32_t* n_launches);
 
 #ifdef __cplusplus
 }

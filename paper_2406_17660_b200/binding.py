@@ -61,6 +61,8 @@ _SIGNATURES = {
     "grass_profile_begin": (c_int, [c_int32]),
     "grass_profile_end": (c_int, [ctypes.POINTER(c_int32), ctypes.POINTER(ctypes.c_float),
                                   ctypes.POINTER(c_int32)]),
+    "grass_profile_end_timeline": (c_int, [ctypes.POINTER(c_int32), ctypes.POINTER(ctypes.c_float),
+                                           ctypes.POINTER(ctypes.c_float), ctypes.POINTER(c_int32)]),
 }
 
 KERNEL_NAMES = ["row_norms", "select", "gather", "project_tc", "splitk_reduce", "project_fp32",
@@ -254,6 +256,20 @@ def grass_device_status(raise_on_error: bool = True):
     if status != 0 and raise_on_error:
         raise GrassError(status, f"device status (detail {detail.value})")
     return status, detail.value
+
+
+def grass_profile_end_timeline():
+    """Returns (launches_seen, [(kernel_name, start_ms, ms), ...]); start_ms counts from the start
+    of the first recorded launch, across streams."""
+    cap = grass_profile_begin.cap
+    kid = (c_int32 * cap)()
+    ms = (ctypes.c_float * cap)()
+    st = (ctypes.c_float * cap)()
+    n = c_int32(0)
+    _check(load_library().grass_profile_end_timeline(kid, ms, st, ctypes.byref(n)),
+           "grass_profile_end_timeline")
+    timed = min(n.value, cap)
+    return n.value, [(KERNEL_NAMES[kid[i]], float(st[i]), float(ms[i])) for i in range(timed)]
 
 
 def grass_selftest_bounded_wait(limit_cycles: int) -> None:

@@ -65,7 +65,15 @@ extern "C" int grass_profile_begin(int32_t max_launches) {
   return GRASS_OK;
 }
 
+extern "C" int grass_profile_end_timeline(int32_t* kernel_id, float* ms, float* start_ms,
+                                          int32_t* n_launches);
+
 extern "C" int grass_profile_end(int32_t* kernel_id, float* ms, int32_t* n_launches) {
+  return grass_profile_end_timeline(kernel_id, ms, nullptr, n_launches);
+}
+
+extern "C" int grass_profile_end_timeline(int32_t* kernel_id, float* ms, float* start_ms,
+                                          int32_t* n_launches) {
   using grass::g_profile;
   if (!g_profile.active) return GRASS_ERR_INVALID_ARG;
   g_profile.active = false;
@@ -78,6 +86,9 @@ extern "C" int grass_profile_end(int32_t* kernel_id, float* ms, int32_t* n_launc
       rc = GRASS_ERR_CUDA;
     if (ms != nullptr) ms[i] = t;
     if (kernel_id != nullptr) kernel_id[i] = g_profile.kid[i];
+    if (start_ms != nullptr &&
+        cudaEventElapsedTime(&start_ms[i], g_profile.start[0], g_profile.start[i]) != cudaSuccess)
+      rc = GRASS_ERR_CUDA;
   }
   if (n_launches != nullptr) *n_launches = g_profile.seen;
   for (int i = 0; i < g_profile.cap; ++i) {
