@@ -289,6 +289,12 @@ def run_gpu(args):
                                                                       device=dev)
         units.append({"obj": obj, "pis": [pi for pi, _ in members], "layers": [l for _, l in members]})
         i = j
+    # Within a step the units are independent, so their order is free.  The first unit's column
+    # gather and the last unit's update have nothing to hide behind: start with the unit that
+    # gathers the fewest bytes (layers x m) and keep the rest in block order.
+    if len(units) > 2:
+        first = min(range(len(units)), key=lambda u: len(units[u]["layers"]) * units[u]["layers"][0].m)
+        units.insert(0, units.pop(first))
     for u, unit in enumerate(units):
         unit["stream"] = streams[u % n_streams]
         for l in unit["layers"]:

@@ -126,18 +126,13 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
 }
 
 template <int MB, int NSLAB, bool PAIR>
-int launch_tc_one(dim3 grid, size_t smem, cudaStream_t s, const TcMaps& maps, const TcParams& p) {
+int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& maps, TcParams p) {
   static bool attr_set[64] = {false};
+  static int max_workers[64] = {0};
   int dev = 0;
   GRASS_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel<MB, NSLAB, PAIR>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        kTcSmemBudget));
-    attr_set[dev] = true;
-  }
+  if (dev < 0 || dev >= 64) return GRASS_ERR_INVALID_ARG;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
   cfg.blockDim = dim3(kTcThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
@@ -148,6 +143,30 @@ int launch_tc_one(dim3 grid, size_t smem, cudaStream_t s, const TcMaps& maps, co
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (!attr_set[dev]) {
+    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel<MB, NSLAB, PAIR>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kTcSmemBudget));
+    // how many workers (CTAs, or CTA pairs) the device holds at once: one per SM / SM pair
+    int workers = 0;
+    if (PAIR) {
+      cfg.gridDim = dim3(2 * kSmCount);
+      GRASS_CUDA_TRY(cudaOccupancyMaxActiveClusters(&workers, project_tc_kernel<MB, NSLAB, PAIR>,
+                                                    &cfg));
+    } else {
+      GRASS_CUDA_TRY(cudaDeviceGetAttribute(&workers, cudaDevAttrMultiProcessorCount, dev));
+    }
+    if (workers < 1) workers = 1;
+    max_workers[dev] = workers;
+    attr_set[dev] = true;
+  }
+  // persistent launch: never more workers than are resident at once, each loops over its tiles
+  p.tiles_x = static_cast<int>(tile_grid.x);
+  p.tiles_y = static_cast<int>(tile_grid.y);
+  p.tiles_z = static_cast<int>(tile_grid.z);
+  const long long n_tiles = static_cast<long long>(tile_grid.x) * tile_grid.y * tile_grid.z;
+  const int workers = n_tiles < max_workers[dev] ? static_cast<int>(n_tiles) : max_workers[dev];
+  cfg.gridDim = dim3(static_cast<unsigned>(PAIR ? 2 * workers : workers));
   {
     ProfileScope prof(GRASS_K_PROJECT_TC, s);
     GRASS_CUDA_TRY(cudaLaunchKernelEx(&cfg, project_tc_kernel<MB, NSLAB, PAIR>, maps, p));
@@ -307,8 +326,9 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   }
   p.ld_out = plan.split_k == 1 ? ldgc : plan.ld_part;
   p.split_stride = plan.split_k == 1 ? 0 : static_cast<long long>(r) * plan.ld_part;
-  dim3 grid(static_cast<unsigned>(plan.n_blocks), static_cast<unsigned>(plan.r_blocks),
-            static_cast<unsigned>(plan.split_k * count));
+  // tile space handed to the persistent kernel (x counts pairs of CTAs in pair mode)
+  dim3 grid(static_cast<unsigned>(plan.pair ? plan.n_blocks / 2 : plan.n_blocks),
+            static_cast<unsigned>(plan.r_blocks), static_cast<unsigned>(plan.split_k * count));
   const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, grid, plan.smem_bytes, s, maps, p);
   if (rc != GRASS_OK) return rc;
   if (norms != nullptr) {

@@ -78,7 +78,9 @@ struct TcMaps {
 struct TcParams {
   int T, n, r;          // logical sizes
   int k_blocks;         // ceil(T / tokens per stage)
-  int split_k;          // gridDim.z
+  int split_k;          // token slices per layer
+  int tiles_x, tiles_y, tiles_z;   // tile space: n-tiles (per pair if PAIR), row blocks,
+                                   // layers * split_k
   // Up to kTcMaxGroup same-shaped layers share one launch: blockIdx.z = group * split_k + split.
   float* out[kTcMaxGroup];        // split_k == 1: Gc, else partials [split][r][ld_out]
   long long ld_out;     // row pitch of out, elements
@@ -118,6 +120,7 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   constexpr int STAGE_BYTES = tc_stage_bytes(MB, A_SLABS);
   constexpr int STAGES = tc_stages(MB, A_SLABS);
   constexpr int UMMA_M = PAIR ? 256 : 128;
+  constexpr int C_STEP = PAIR ? 256 : 128;   // columns between this CTA's consecutive blocks
   static_assert(MB * R_CTA <= 512, "accumulators exceed TMEM");
   static_assert(N_SLABS <= 32, "one producer lane per slab");
   static_assert(!PAIR || NSLAB % 2 == 0, "a CTA pair splits the selected rows in halves of 64k");
@@ -125,27 +128,42 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kTcMaxStages];
   __shared__ __align__(8) uint64_t bar_empty[kTcMaxStages];
-  __shared__ __align__(8) uint64_t bar_accum;
+  __shared__ __align__(8) uint64_t bar_accum;       // accumulators of the current tile complete
+  __shared__ __align__(8) uint64_t bar_tmem_free;   // every epilogue warp has read them out
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                               ~static_cast<uintptr_t>(1023));
-  // PAIR: CTA `rank` of pair `blockIdx.x / 2` owns, for each of its MB blocks, the 128 columns
-  // pair_base + (mb * 2 + rank) * 128; otherwise the CTA owns MB consecutive blocks.
   const int rank = PAIR ? static_cast<int>(ptx::cluster_ctarank()) : 0;
-  const int c_base = PAIR ? (blockIdx.x >> 1) * (2 * MB * 128) + rank * 128 : blockIdx.x * (MB * 128);
-  constexpr int C_STEP = PAIR ? 256 : 128;   // columns between this CTA's consecutive blocks
-  const int r0 = blockIdx.y * R_CTA;
-  // this CTA's token blocks: [kb_begin, kb_begin + kb_count)
+  // Persistent workers: a worker (a CTA, or a CTA pair) takes the tiles w, w + W, w + 2W, ... of
+  // the linear tile space [tile_x fastest, then row block, then (layer, token slice)], i.e. the
+  // same order a plain grid would be dispatched in, so concurrent workers still sweep the tokens
+  // together.  The grid never exceeds what is resident at once: the whole grid is dispatched
+  // immediately and kernels of other streams can be scheduled beside it.
+  const int n_workers = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+  const int worker = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int n_tiles = p.tiles_x * p.tiles_y * p.tiles_z;
   const int kb_per = p.k_blocks / p.split_k, kb_rem = p.k_blocks % p.split_k;
-  const int grp = blockIdx.z / p.split_k;          // which layer of the group
-  const int z = blockIdx.z - grp * p.split_k;      // which token slice
-  const CUtensorMap* tmX = &maps.x[grp];
-  const CUtensorMap* tmA = &maps.a[grp];
-  const int kb_begin = z * kb_per + (z < kb_rem ? z : kb_rem);
-  const int kb_count = kb_per + (z < kb_rem ? 1 : 0);
+
+  // decode a linear tile index (identical in every role)
+  struct Tile { int c_base, r0, grp, z, kb_begin, kb_count; };
+  auto decode = [&](int L) {
+    Tile t;
+    const int bx = L % p.tiles_x;
+    const int rest = L / p.tiles_x;
+    const int by = rest % p.tiles_y, bz = rest / p.tiles_y;
+    // PAIR: CTA `rank` of the pair owns, for each of its MB blocks, the 128 columns
+    // pair_base + (mb * 2 + rank) * 128; otherwise the CTA owns MB consecutive blocks.
+    t.c_base = PAIR ? bx * (2 * MB * 128) + rank * 128 : bx * (MB * 128);
+    t.r0 = by * R_CTA;
+    t.grp = bz / p.split_k;                 // which layer of the group
+    t.z = bz - t.grp * p.split_k;           // which token slice
+    t.kb_begin = t.z * kb_per + (t.z < kb_rem ? t.z : kb_rem);
+    t.kb_count = kb_per + (t.z < kb_rem ? 1 : 0);
+    return t;
+  };
 
   if (threadIdx.x == 0) {
     s_abort = 0;
@@ -155,9 +173,10 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
       ptx::mbar_init(&bar_empty[s], 1);
     }
     ptx::mbar_init(&bar_accum, 1);
+    ptx::mbar_init(&bar_tmem_free, (kTcThreads / 32 - 2) * (PAIR ? 2 : 1));
     ptx::fence_mbar_init();
-    ptx::prefetch_tensormap(tmX);
-    ptx::prefetch_tensormap(tmA);
+    ptx::prefetch_tensormap(&maps.x[0]);
+    ptx::prefetch_tensormap(&maps.a[0]);
   }
   if (warp == 1) {
     if (PAIR) {
@@ -177,44 +196,48 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   if (warp == 0) {
     // ================= TMA producer: one lane per slab =================
     const bool is_x = lane < X_SLABS;
-    const CUtensorMap* map = is_x ? tmX : tmA;
-    int xcoord;
-    if (is_x) {
-      xcoord = c_base + (lane >> 1) * C_STEP + (lane & 1) * 64;
-    } else if (PAIR) {
-      // slab a of this CTA: 256-row chunk a/2 of the tile, this CTA's half of it
-      const int a = lane - X_SLABS, q = a >> 1;
-      const int wq = R_CTA - 256 * q < 256 ? R_CTA - 256 * q : 256;
-      xcoord = r0 + 256 * q + rank * (wq >> 1) + (a & 1) * 64;
-    } else {
-      xcoord = r0 + (lane - X_SLABS) * 64;
-    }
     uint8_t* my_dst = tiles + lane * kTcSlabBytes;
-    int tok = kb_begin * kTcBK;
     int s = 0, issued = 0;
     uint32_t ph = 0;
-    for (int it = 0; it < kb_count; ++it) {
-      int ok = 1;
-      if (lane == 0) {
-        ok = ptx::mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kTcWaitLimit) ? 1 : 0;
-        if (ok) {
-          // PAIR: the even CTA's barrier collects the bytes of both CTAs
-          if (!PAIR) ptx::mbar_arrive_expect_tx(&bar_full[s], STAGE_BYTES);
-          else if (rank == 0) ptx::mbar_arrive_expect_tx(&bar_full[s], 2 * STAGE_BYTES);
-        } else {
-          if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 100 + s);
-          *abort_flag = 1;
+    bool alive = true;
+    for (int L = worker; L < n_tiles && alive; L += n_workers) {
+      const Tile t = decode(L);
+      const CUtensorMap* map = is_x ? &maps.x[t.grp] : &maps.a[t.grp];
+      int xcoord;
+      if (is_x) {
+        xcoord = t.c_base + (lane >> 1) * C_STEP + (lane & 1) * 64;
+      } else if (PAIR) {
+        // slab a of this CTA: 256-row chunk a/2 of the tile, this CTA's half of it
+        const int a = lane - X_SLABS, q = a >> 1;
+        const int wq = R_CTA - 256 * q < 256 ? R_CTA - 256 * q : 256;
+        xcoord = t.r0 + 256 * q + rank * (wq >> 1) + (a & 1) * 64;
+      } else {
+        xcoord = t.r0 + (lane - X_SLABS) * 64;
+      }
+      int tok = t.kb_begin * kTcBK;
+      for (int it = 0; it < t.kb_count; ++it) {
+        int ok = 1;
+        if (lane == 0) {
+          ok = ptx::mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kTcWaitLimit) ? 1 : 0;
+          if (ok) {
+            // PAIR: the even CTA's barrier collects the bytes of both CTAs
+            if (!PAIR) ptx::mbar_arrive_expect_tx(&bar_full[s], STAGE_BYTES);
+            else if (rank == 0) ptx::mbar_arrive_expect_tx(&bar_full[s], 2 * STAGE_BYTES);
+          } else {
+            if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 100 + s);
+            *abort_flag = 1;
+          }
         }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) { alive = false; break; }
+        if (lane < N_SLABS) {
+          if (PAIR) ptx::tma_load_2d_pair(my_dst + s * STAGE_BYTES, map, xcoord, tok, &bar_full[s]);
+          else ptx::tma_load_2d(my_dst + s * STAGE_BYTES, map, xcoord, tok, &bar_full[s]);
+        }
+        tok += kTcBK;
+        ++issued;
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      if (lane < N_SLABS) {
-        if (PAIR) ptx::tma_load_2d_pair(my_dst + s * STAGE_BYTES, map, xcoord, tok, &bar_full[s]);
-        else ptx::tma_load_2d(my_dst + s * STAGE_BYTES, map, xcoord, tok, &bar_full[s]);
-      }
-      tok += kTcBK;
-      issued = it + 1;
-      if (++s == STAGES) { s = 0; ph ^= 1u; }
     }
     if (lane == 0 && *abort_flag != 0 && rank == 0) {
       // let the copies already issued land before the CTA gives its smem back
@@ -230,87 +253,106 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
       const uint64_t desc0 = ptx::smem_desc_mn_sw128(ptx::smem_u32(tiles), LBO, SBO);
       bool ok = true;
       int s = 0;
-      uint32_t ph = 0;
-      for (int it = 0; it < kb_count; ++it) {
-        if (!ptx::mbar_wait_bounded(&bar_full[s], ph, abort_flag, kTcWaitLimit)) {
-          if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 200 + s);
-          *abort_flag = 1;
-          ok = false;
-          break;
+      uint32_t ph = 0, tile_ph = 0;
+      bool first_tile = true;
+      for (int L = worker; L < n_tiles && ok; L += n_workers) {
+        const Tile t = decode(L);
+        if (!first_tile) {
+          // the accumulators are reused: the epilogue warps (of both CTAs) must have read the
+          // previous tile out of TMEM before the first MMA of this one overwrites it
+          if (!ptx::mbar_wait_bounded(&bar_tmem_free, tile_ph ^ 1u, abort_flag, kTcWaitLimit)) {
+            if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 250);
+            *abort_flag = 1;
+            ok = false;
+            break;
+          }
+          ptx::fence_tc_after_sync();
         }
-        ptx::fence_tc_after_sync();
-        const uint64_t dstage = desc0 + static_cast<uint64_t>((s * STAGE_BYTES) >> 4);
+        first_tile = false;
+        for (int it = 0; it < t.kb_count; ++it) {
+          if (!ptx::mbar_wait_bounded(&bar_full[s], ph, abort_flag, kTcWaitLimit)) {
+            if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 200 + s);
+            *abort_flag = 1;
+            ok = false;
+            break;
+          }
+          ptx::fence_tc_after_sync();
+          const uint64_t dstage = desc0 + static_cast<uint64_t>((s * STAGE_BYTES) >> 4);
 #pragma unroll
-        for (int ks = 0; ks < kTcBK / 16; ++ks) {
-          const uint32_t acc = (it | ks) != 0 ? 1u : 0u;
+          for (int ks = 0; ks < kTcBK / 16; ++ks) {
+            const uint32_t acc = (it | ks) != 0 ? 1u : 0u;
 #pragma unroll
-          for (int mb = 0; mb < MB; ++mb) {
-            // 16 tokens = 2 groups of 8 rows = 2 * SBO bytes into every slab
-            const uint64_t adesc = dstage + ((mb * 2 * kTcSlabBytes + ks * 2 * SBO) >> 4);
+            for (int mb = 0; mb < MB; ++mb) {
+              // 16 tokens = 2 groups of 8 rows = 2 * SBO bytes into every slab
+              const uint64_t adesc = dstage + ((mb * 2 * kTcSlabBytes + ks * 2 * SBO) >> 4);
 #pragma unroll
-            for (int j = 0; j < R_CTA; j += 256) {
-              constexpr int kFull = 256;
-              const int ncols = R_CTA - j < kFull ? R_CTA - j : kFull;
-              // slabs of this 256-row chunk in a CTA's stage: 4 per chunk, or 2 when split over a pair
-              const int bslab = PAIR ? (j / 256) * 2 : j / 64;
-              const uint64_t bdesc =
-                  dstage + ((X_SLABS * kTcSlabBytes + bslab * kTcSlabBytes + ks * 2 * SBO) >> 4);
-              const uint32_t idesc = ptx::idesc_bf16_mn_mn(UMMA_M, static_cast<uint32_t>(ncols));
-              const uint32_t d = tmem_base + static_cast<uint32_t>(mb * R_CTA + j);
-              if (PAIR) ptx::mma_bf16_pair(d, adesc, bdesc, idesc, acc);
-              else ptx::mma_bf16(d, adesc, bdesc, idesc, acc);
+              for (int j = 0; j < R_CTA; j += 256) {
+                constexpr int kFull = 256;
+                const int ncols = R_CTA - j < kFull ? R_CTA - j : kFull;
+                // slabs of this 256-row chunk in a CTA's stage: 4, or 2 when split over a pair
+                const int bslab = PAIR ? (j / 256) * 2 : j / 64;
+                const uint64_t bdesc =
+                    dstage + ((X_SLABS * kTcSlabBytes + bslab * kTcSlabBytes + ks * 2 * SBO) >> 4);
+                const uint32_t idesc = ptx::idesc_bf16_mn_mn(UMMA_M, static_cast<uint32_t>(ncols));
+                const uint32_t d = tmem_base + static_cast<uint32_t>(mb * R_CTA + j);
+                if (PAIR) ptx::mma_bf16_pair(d, adesc, bdesc, idesc, acc);
+                else ptx::mma_bf16(d, adesc, bdesc, idesc, acc);
+              }
             }
           }
+          // frees the stage (in both CTAs if PAIR) once these MMAs have read it
+          if (PAIR) ptx::mma_commit_pair(&bar_empty[s]); else ptx::mma_commit(&bar_empty[s]);
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
-        // frees the stage (in both CTAs if PAIR) once these MMAs have read it
-        if (PAIR) ptx::mma_commit_pair(&bar_empty[s]); else ptx::mma_commit(&bar_empty[s]);
-        if (++s == STAGES) { s = 0; ph ^= 1u; }
+        // accumulators of this tile complete (or: everything issued so far is done)
+        if (PAIR) ptx::mma_commit_pair(&bar_accum); else ptx::mma_commit(&bar_accum);
+        if (!ok) ptx::mbar_wait_bounded(&bar_accum, tile_ph, nullptr, kTcDrainLimit);
+        tile_ph ^= 1u;
       }
-      // accumulators complete (or: everything issued is done)
-      if (PAIR) ptx::mma_commit_pair(&bar_accum); else ptx::mma_commit(&bar_accum);
-      if (!ok) ptx::mbar_wait_bounded(&bar_accum, 0, nullptr, kTcDrainLimit);
     }
   } else {
     // ================= epilogue: TMEM -> registers -> global =================
     const int q = warp & 3;             // TMEM lane quarter this warp may touch
     const int half = (warp - 2) >> 2;   // which of the quarter's two warps
-    bool ok = kb_count > 0;
-    if (ok) {
-      // one polling lane per warp, with back-off: this wait lasts the whole main loop
+    uint32_t tile_ph = 0;
+    bool alive = true;
+    for (int L = worker; L < n_tiles && alive; L += n_workers) {
+      const Tile t = decode(L);
+      // one polling lane per warp, with back-off: this wait lasts a whole main loop
       int got = 1;
       if (lane == 0) {
-        got = ptx::mbar_wait_bounded(&bar_accum, 0, abort_flag, kTcWaitLimit, 128) ? 1 : 0;
+        got = ptx::mbar_wait_bounded(&bar_accum, tile_ph, abort_flag, kTcWaitLimit, 128) ? 1 : 0;
         if (!got) {
           if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 300 + warp);
           *abort_flag = 1;
         }
       }
-      ok = __shfl_sync(0xffffffffu, got, 0) != 0;
-    }
-    if (ok && *abort_flag == 0) {
+      got = __shfl_sync(0xffffffffu, got, 0);
+      if (!got || *abort_flag != 0) { alive = false; break; }
+      tile_ph ^= 1u;
       ptx::fence_tc_after_sync();
-      float* out = p.out[grp] + static_cast<long long>(z) * p.split_stride;
-      const float* rho = p.rho[grp];
+      float* out = p.out[t.grp] + static_cast<long long>(t.z) * p.split_stride;
+      const float* rho = p.rho[t.grp];
       const bool scale = p.split_k == 1 && rho != nullptr;
       const long long ld = p.ld_out;
 #pragma unroll 1
       for (int chunk = half; chunk < MB * (R_CTA / 32); chunk += 2) {
         const int mb = chunk / (R_CTA / 32);
         const int j = (chunk % (R_CTA / 32)) * 32;
-        const int row0 = r0 + j;
+        const int row0 = t.r0 + j;
         if (row0 >= p.r) continue;      // uniform: padding rows
         uint32_t v[32];
         ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                static_cast<uint32_t>(mb * R_CTA + j), v);
         ptx::tmem_ld_wait();
-        const int c = c_base + mb * C_STEP + q * 32 + lane;
+        const int c = t.c_base + mb * C_STEP + q * 32 + lane;
         if (p.norm_part != nullptr) {
           // fused row norms of the dense gradient (columns past n were zero-filled by TMA)
           float sq[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) sq[i] = __uint_as_float(v[i]) * __uint_as_float(v[i]);
           const float total = warp_transpose_sum(sq, lane);
-          const int g = (c_base + mb * C_STEP + q * 32) >> 5;
+          const int g = (t.c_base + mb * C_STEP + q * 32) >> 5;
           if (row0 + lane < p.r && (g << 5) < p.n) p.norm_part[g * p.ld_norm + row0 + lane] = total;
           continue;
         }
@@ -332,6 +374,10 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
           }
         }
       }
+      // this warp's reads of TMEM are complete (tcgen05.wait::ld above): tell the MMA issuer
+      ptx::fence_tc_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_leader(&bar_tmem_free);
     }
   }
   __syncwarp();
