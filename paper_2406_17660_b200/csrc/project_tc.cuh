@@ -16,6 +16,11 @@
 // column = j, so the epilogue's tcgen05.ld hands each warp 32 consecutive c for
 // one j per register: every store instruction writes 128 contiguous bytes.
 //
+// The kernel is persistent: at most one CTA (pair) per SM (pair), each looping over tiles, so
+// TMEM, barriers and the TMA ring are set up once and the producer keeps the ring full across
+// tile boundaries; a "TMEM free" barrier returns the accumulators from the epilogue warps to
+// the MMA issuer between tiles.
+//
 // Warp roles (320 threads): warp 0 = TMA producer (one lane per slab), warp 1 =
 // TMEM owner + single-thread MMA issuer, warps 2..9 = epilogue (warp w reads
 // TMEM lanes 32*(w%4)..+31; the two warps of a lane quarter alternate over the
