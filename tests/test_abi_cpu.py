@@ -63,6 +63,16 @@ def test_argument_errors_are_returned_without_a_device(lib):
                                    null) == 1                                # step < 1
     assert lib.grass_subspace_adam(fake, 8, fake, fake, fake, 8, 4, 8, 1e-3, 1.0, 0.999, 1e-8, 1,
                                    null) == 1                                # beta1 = 1
+    # empty problems are argument errors, not launches
+    assert lib.grass_row_norms(fake, 0, 0, 4, 4, fake, null) == 1
+    assert lib.grass_project_grad(fake, 8, fake, 8, 1, 0, 8, 8, fake, null, 4, fake, 8, null, 0,
+                                  null) == 1                                 # T = 0
+    assert lib.grass_project_grad(fake, 8, fake, 8, 1, 16, 8, 8, fake, null, 0, fake, 8, null, 0,
+                                  null) == 1                                 # r = 0
+    assert lib.grass_subspace_adam(fake, 8, fake, fake, fake, 8, 0, 8, 1e-3, 0.9, 0.999, 1e-8, 1,
+                                   null) == 1                                # r = 0
+    assert lib.grass_grad_row_norms(fake, 8, fake, 8, 1, 0, 8, 8, fake, null, 0, null) == 1
+    assert lib.grass_selftest_bounded_wait(0, null) == 1
     assert lib.grass_scatter_update(fake, 1, 8, 8, 8, fake, 8, null, null, 4, 0.25, null) == 1
     assert lib.grass_scatter_update(fake, 5, 8, 8, 8, fake, 8, fake, null, 4, 0.25, null) == 3
 
