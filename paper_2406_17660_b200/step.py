@@ -129,7 +129,8 @@ class GrassLayerGroup:
         self._inputs = {}
 
     def _input_arrays(self, dYs, Xs):
-        key = tuple(t.data_ptr() for t in dYs) + tuple(t.data_ptr() for t in Xs)
+        key = tuple((t.data_ptr(), t.shape[0], t.stride(0)) for t in dYs) + \
+            tuple((t.data_ptr(), t.shape[0], t.stride(0)) for t in Xs)
         hit = self._inputs.get(key)
         if hit is None:
             if len(self._inputs) > 64:
