@@ -472,7 +472,7 @@ def run_gpu(args):
     # ---- the oracle on the host cores, rank 0 of a single-GPU run only ----
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        T_gen = min(wl.T, 8192)
+        T_gen = min(wl.T, 16384)            # about 10 s of oracle work on 16 host threads
         ins = [(syn.to_f32_numpy(d[:T_gen]), syn.to_f32_numpy(x[:T_gen])) for d, x in block_in]
         Ws = [syn.to_f32_numpy(layers[pi][1].W) for pi in range(len(wl.shapes))]
         sub = workloads.get(args.workload, r=args.rank, T=T_gen, layers=args.layers)
