@@ -125,7 +125,7 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
   return true;
 }
 
-template <int MB, int NSLAB, bool PAIR>
+template <int MB, int NSLAB, bool PAIR, bool FUSED>
 int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& maps, TcParams p) {
   static bool attr_set[64] = {false};
   static int max_workers[64] = {0};
@@ -133,7 +133,7 @@ int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& map
   GRASS_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return GRASS_ERR_INVALID_ARG;
   cudaLaunchConfig_t cfg = {};
-  cfg.blockDim = dim3(kTcThreads);
+  cfg.blockDim = dim3(FUSED ? kTcThreads + kTcGatherThreads : kTcThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
@@ -144,14 +144,14 @@ int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& map
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (!attr_set[dev]) {
-    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel<MB, NSLAB, PAIR>,
+    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel<MB, NSLAB, PAIR, FUSED>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kTcSmemBudget));
     // how many workers (CTAs, or CTA pairs) the device holds at once: one per SM / SM pair
     int workers = 0;
     if (PAIR) {
       cfg.gridDim = dim3(2 * kSmCount);
-      GRASS_CUDA_TRY(cudaOccupancyMaxActiveClusters(&workers, project_tc_kernel<MB, NSLAB, PAIR>,
+      GRASS_CUDA_TRY(cudaOccupancyMaxActiveClusters(&workers, project_tc_kernel<MB, NSLAB, PAIR, FUSED>,
                                                     &cfg));
     } else {
       GRASS_CUDA_TRY(cudaDeviceGetAttribute(&workers, cudaDevAttrMultiProcessorCount, dev));
@@ -169,25 +169,34 @@ int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& map
   cfg.gridDim = dim3(static_cast<unsigned>(PAIR ? 2 * workers : workers));
   {
     ProfileScope prof(GRASS_K_PROJECT_TC, s);
-    GRASS_CUDA_TRY(cudaLaunchKernelEx(&cfg, project_tc_kernel<MB, NSLAB, PAIR>, maps, p));
+    GRASS_CUDA_TRY(cudaLaunchKernelEx(&cfg, project_tc_kernel<MB, NSLAB, PAIR, FUSED>, maps, p));
   }
   return GRASS_OK;
 }
 
 // (MB, NSLAB) with MB * 64 * NSLAB <= 512 TMEM columns; pairs need an even NSLAB.
-int launch_tc(int MB, int nslab, bool pair, dim3 grid, size_t smem, cudaStream_t s,
+int launch_tc(int MB, int nslab, bool pair, bool fused, dim3 grid, size_t smem, cudaStream_t s,
               const TcMaps& maps, const TcParams& p) {
 #define GRASS_TC_CASE(mb, ns)                                                                  \
-  if (MB == mb && nslab == ns && !pair)                                                        \
-    return launch_tc_one<mb, ns, false>(grid, smem, s, maps, p)
+  if (MB == mb && nslab == ns && !pair && !fused)                                              \
+    return launch_tc_one<mb, ns, false, false>(grid, smem, s, maps, p)
 #define GRASS_TC_PAIR(mb, ns)                                                                  \
-  if (MB == mb && nslab == ns && pair) return launch_tc_one<mb, ns, true>(grid, smem, s, maps, p)
+  if (MB == mb && nslab == ns && pair && !fused)                                               \
+    return launch_tc_one<mb, ns, true, false>(grid, smem, s, maps, p)
+#define GRASS_TC_FUSED(mb, ns, pr)                                                             \
+  if (MB == mb && nslab == ns && pair == pr && fused)                                          \
+    return launch_tc_one<mb, ns, pr, true>(grid, smem, s, maps, p)
   GRASS_TC_CASE(1, 1); GRASS_TC_CASE(1, 2); GRASS_TC_CASE(1, 3); GRASS_TC_CASE(1, 4);
   GRASS_TC_CASE(1, 5); GRASS_TC_CASE(1, 6); GRASS_TC_CASE(1, 7); GRASS_TC_CASE(1, 8);
   GRASS_TC_CASE(2, 1); GRASS_TC_CASE(2, 2); GRASS_TC_CASE(2, 3); GRASS_TC_CASE(2, 4);
   GRASS_TC_CASE(4, 1); GRASS_TC_CASE(4, 2);
   GRASS_TC_PAIR(1, 2); GRASS_TC_PAIR(1, 4); GRASS_TC_PAIR(1, 6); GRASS_TC_PAIR(1, 8);
   GRASS_TC_PAIR(2, 2); GRASS_TC_PAIR(2, 4); GRASS_TC_PAIR(4, 2);
+  // in-kernel gather: at most 128 selected rows per tile
+  GRASS_TC_FUSED(1, 1, false); GRASS_TC_FUSED(2, 1, false); GRASS_TC_FUSED(4, 1, false);
+  GRASS_TC_FUSED(1, 2, false); GRASS_TC_FUSED(2, 2, false); GRASS_TC_FUSED(4, 2, false);
+  GRASS_TC_FUSED(1, 2, true); GRASS_TC_FUSED(2, 2, true); GRASS_TC_FUSED(4, 2, true);
+#undef GRASS_TC_FUSED
 #undef GRASS_TC_CASE
 #undef GRASS_TC_PAIR
   return GRASS_ERR_UNSUPPORTED;
@@ -256,8 +265,21 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   }
   const TcPlan plan = norms != nullptr ? make_norms_plan(T, n, r) : make_plan(T, n, r, false, count);
   const bool fused_norms = norms != nullptr && plan.split_k == 1;
+  // In-kernel gather: the GEMM's own warps pick the selected columns out of dY.  It pays when a
+  // tile holds at most 128 rows (the load unit keeps up) and at most two CTAs (pairs) share a
+  // token slice (each of them gathers for itself): then the copy pre-pass, its launch and the
+  // round trip of the gathered operand through HBM all disappear.  Measured: 60M q,k,v,o group
+  // (m = 512, r = 128) step 253 -> 274 TFLOP/s; at m = 2048, r = 128 the sparser pick makes the
+  // in-kernel loads the bottleneck (471 -> 379 TFLOP/s), hence the density condition
+  // (32 neighbouring picks span 64 / density bytes = 0.5 / density 128-byte lines).
+  static const bool no_fuse = getenv("GRASS_TC_NO_FUSED_GATHER") != nullptr;   // diagnostic
+  const int tiles_x = plan.pair ? plan.n_blocks / 2 : plan.n_blocks;
+  static const int max_tiles_x = getenv("GRASS_TC_FUSED_MAX_TILES") != nullptr
+                                     ? atoi(getenv("GRASS_TC_FUSED_MAX_TILES")) : 2;   // diagnostic
+  const bool fused_gather = gather && !no_fuse && plan.r_cta <= 128 && tiles_x <= max_tiles_x &&
+                            static_cast<int64_t>(r) * 12 >= m;  // a 32-lane load then spans <= 6 lines
   const size_t per_layer = fused_norms ? norm_part_bytes(m, n)
-                                       : (gather ? plan.ag_bytes : 0) + plan.part_bytes;
+                                       : (gather && !fused_gather ? plan.ag_bytes : 0) + plan.part_bytes;
   const size_t need = per_layer * count;
   if (need > 0 && (ws == nullptr || !aligned_to(ws, 256) || ws_bytes < need))
     return GRASS_ERR_WORKSPACE;
@@ -271,7 +293,12 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   for (int g = 0; g < count; ++g) {
     char* wsp = static_cast<char*>(ws) + per_layer * g;
     if (!make_map(&maps.x[g], X[g], T, n, ldx, plan.bk)) return GRASS_ERR_CUDA;
-    if (gather) {
+    if (fused_gather) {
+      gg.dY[g] = static_cast<const __nv_bfloat16*>(dY[g]);
+      gg.idx[g] = idx[g];
+      gg.Ag[g] = nullptr;
+      maps.a[g] = maps.x[g];          // unused by the kernel
+    } else if (gather) {
       gg.dY[g] = static_cast<const __nv_bfloat16*>(dY[g]);
       gg.idx[g] = idx[g];
       gg.Ag[g] = reinterpret_cast<__nv_bfloat16*>(wsp);
@@ -287,7 +314,7 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
     maps.a[g] = maps.a[0];
     gg.dY[g] = nullptr; gg.idx[g] = nullptr; gg.Ag[g] = nullptr;
   }
-  if (gather) {
+  if (gather && !fused_gather) {
     ProfileScope prof(GRASS_K_GATHER, s);
     const int ni = plan.r_pad >= 256 ? 8 : plan.r_pad / 32;   // r_pad is a multiple of 64
     dim3 ggrid(static_cast<unsigned>((plan.r_pad + 32 * ni - 1) / (32 * ni)),
@@ -307,13 +334,20 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   p.split_k = plan.split_k;
   p.status = status;
   p.norm_part = fused_norms ? part[0] : nullptr;
+  for (int g = 0; g < kTcMaxGroup; ++g) {
+    const int gi = g < count ? g : 0;
+    p.dY[g] = fused_gather ? gg.dY[gi] : nullptr;
+    p.idx[g] = fused_gather ? gg.idx[gi] : nullptr;
+  }
+  p.lddy = lddy;
+  p.m = static_cast<int>(m);
   p.ld_norm = static_cast<long long>(round_up(static_cast<size_t>(m), 32));
   static const bool debug_plan = getenv("GRASS_DEBUG_PLAN") != nullptr;   // read once
   if (debug_plan)
     fprintf(stderr, "grass plan T=%lld n=%lld r=%d x%d: r_cta=%d r_blocks=%d MB=%d n_blocks=%d "
-                    "split_k=%d stages=%d pair=%d\n", static_cast<long long>(T),
+                    "split_k=%d stages=%d pair=%d fused_gather=%d\n", static_cast<long long>(T),
             static_cast<long long>(n), r, count, plan.r_cta, plan.r_blocks, plan.MB, plan.n_blocks,
-            plan.split_k, plan.stages, plan.pair ? 1 : 0);
+            plan.split_k, plan.stages, plan.pair ? 1 : 0, fused_gather ? 1 : 0);
   for (int g = 0; g < kTcMaxGroup; ++g) {
     const int gi = g < count ? g : 0;
     if (plan.split_k == 1) {
@@ -329,7 +363,7 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   // tile space handed to the persistent kernel (x counts pairs of CTAs in pair mode)
   dim3 grid(static_cast<unsigned>(plan.pair ? plan.n_blocks / 2 : plan.n_blocks),
             static_cast<unsigned>(plan.r_blocks), static_cast<unsigned>(plan.split_k * count));
-  const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, grid, plan.smem_bytes, s, maps, p);
+  const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, fused_gather, grid, plan.smem_bytes, s, maps, p);
   if (rc != GRASS_OK) return rc;
   if (norms != nullptr) {
     ProfileScope prof(GRASS_K_ROW_NORMS, s);

@@ -52,6 +52,7 @@ namespace grass {
 // issue); with 64 tokens that cost is spread over twice as many MMAs (234 -> 193 us on the
 // LLaMA-7B q shape).  A slab is [BK tokens][64 bf16].
 constexpr int kTcThreads = 320;
+constexpr int kTcGatherThreads = 256;   // extra warps of the in-kernel gather variant
 constexpr int kTcMaxStages = 8;
 constexpr int kTcSmemBudget = 227 * 1024 - 1024;  // dynamic part; the rest holds the barriers
 constexpr long long kTcWaitLimit = 2000000000LL;  // SM clocks (~1 s)
@@ -91,6 +92,11 @@ struct TcParams {
   long long ld_out;     // row pitch of out, elements
   long long split_stride;  // elements between partials of consecutive splits
   const float* rho[kTcMaxGroup];  // applied here only when split_k == 1 (entries may be NULL)
+  // in-kernel gather variant: the selected columns are picked straight out of dY
+  const __nv_bfloat16* dY[kTcMaxGroup];
+  const int32_t* idx[kTcMaxGroup];
+  long long lddy;
+  int m;
   float* norm_part;     // non-NULL: row-norm mode.  Nothing of D is stored; instead
                         // norm_part[g * ld_norm + j] = sum of D[j, c]^2 over the 32 columns c of group g
   long long ld_norm;
@@ -113,8 +119,8 @@ __device__ __forceinline__ float warp_transpose_sum(float (&x)[32], int lane) {
   return x[0];
 }
 
-template <int MB, int NSLAB, bool PAIR>
-__global__ void __launch_bounds__(kTcThreads, 1)
+template <int MB, int NSLAB, bool PAIR, bool FUSED>
+__global__ void __launch_bounds__(kTcThreads + kTcGatherThreads, 1)
 project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   constexpr int R_CTA = 64 * NSLAB;          // selected rows per CTA tile (per pair if PAIR)
   constexpr int X_SLABS = 2 * MB;
@@ -123,6 +129,11 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   constexpr int kTcBK = tc_bk(MB, A_SLABS);           // tokens per stage
   constexpr int kTcSlabBytes = kTcBK * 128;
   constexpr int STAGE_BYTES = tc_stage_bytes(MB, A_SLABS);
+  // FUSED: the gathered operand is not copied by TMA but picked out of dY by the gather warps,
+  // so only the X slabs are TMA traffic; every gather warp of the pair reports to "full"
+  constexpr int TMA_SLABS = FUSED ? X_SLABS : N_SLABS;
+  constexpr int TMA_BYTES = TMA_SLABS * kTcSlabBytes;
+  constexpr int FULL_ARRIVALS = 1 + (FUSED ? (kTcGatherThreads / 32) * (PAIR ? 2 : 1) : 0);
   constexpr int STAGES = tc_stages(MB, A_SLABS);
   constexpr int UMMA_M = PAIR ? 256 : 128;
   constexpr int C_STEP = PAIR ? 256 : 128;   // columns between this CTA's consecutive blocks
@@ -174,7 +185,7 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     s_abort = 0;
 #pragma unroll
     for (int s = 0; s < STAGES; ++s) {
-      ptx::mbar_init(&bar_full[s], 1);
+      ptx::mbar_init(&bar_full[s], FULL_ARRIVALS);
       ptx::mbar_init(&bar_empty[s], 1);
     }
     ptx::mbar_init(&bar_accum, 1);
@@ -226,8 +237,8 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
           ok = ptx::mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kTcWaitLimit) ? 1 : 0;
           if (ok) {
             // PAIR: the even CTA's barrier collects the bytes of both CTAs
-            if (!PAIR) ptx::mbar_arrive_expect_tx(&bar_full[s], STAGE_BYTES);
-            else if (rank == 0) ptx::mbar_arrive_expect_tx(&bar_full[s], 2 * STAGE_BYTES);
+            if (!PAIR) ptx::mbar_arrive_expect_tx(&bar_full[s], TMA_BYTES);
+            else if (rank == 0) ptx::mbar_arrive_expect_tx(&bar_full[s], 2 * TMA_BYTES);
           } else {
             if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 100 + s);
             *abort_flag = 1;
@@ -235,7 +246,7 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) { alive = false; break; }
-        if (lane < N_SLABS) {
+        if (lane < TMA_SLABS) {
           if (PAIR) ptx::tma_load_2d_pair(my_dst + s * STAGE_BYTES, map, xcoord, tok, &bar_full[s]);
           else ptx::tma_load_2d(my_dst + s * STAGE_BYTES, map, xcoord, tok, &bar_full[s]);
         }
@@ -275,7 +286,7 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         }
         first_tile = false;
         for (int it = 0; it < t.kb_count; ++it) {
-          if (!ptx::mbar_wait_bounded(&bar_full[s], ph, abort_flag, kTcWaitLimit)) {
+          if (!ptx::mbar_wait_bounded(&bar_full[s], ph, abort_flag, kTcWaitLimit, 0, FUSED && PAIR)) {
             if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 200 + s);
             *abort_flag = 1;
             ok = false;
@@ -313,6 +324,94 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         if (PAIR) ptx::mma_commit_pair(&bar_accum); else ptx::mma_commit(&bar_accum);
         if (!ok) ptx::mbar_wait_bounded(&bar_accum, tile_ph, nullptr, kTcDrainLimit);
         tile_ph ^= 1u;
+      }
+    }
+  } else if (FUSED && warp >= kTcThreads / 32) {
+    // ================= gather warps (FUSED): dY[t, idx[j]] -> swizzled B-operand slabs =================
+    // Warp g takes tokens g, g + GW, ... of the stage; lane l carries j = slab base + l and + 32:
+    // one load instruction reads 32 neighbouring selected columns of one dY row.  The bytes go
+    // where a TMA box {64, BK} with the 128-byte swizzle would put them: row t of a slab is 128
+    // bytes, its 16-byte chunks XOR-ed with (t mod 8).
+    const int g = warp - kTcThreads / 32;
+    constexpr int GW = kTcGatherThreads / 32;
+    int s = 0;
+    uint32_t ph = 0;
+    bool alive = true;
+    for (int L = worker; L < n_tiles && alive; L += n_workers) {
+      const Tile t = decode(L);
+      const unsigned short* src = reinterpret_cast<const unsigned short*>(p.dY[t.grp]);
+      const int32_t* idx = p.idx[t.grp];
+      int rows[A_SLABS][2];
+#pragma unroll
+      for (int a = 0; a < A_SLABS; ++a) {
+        int jb;
+        if (PAIR) {
+          const int q2 = a >> 1;
+          const int wq = R_CTA - 256 * q2 < 256 ? R_CTA - 256 * q2 : 256;
+          jb = t.r0 + 256 * q2 + rank * (wq >> 1) + (a & 1) * 64;
+        } else {
+          jb = t.r0 + a * 64;
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int j = jb + 32 * h + lane;
+          int row = -1;
+          if (j < p.r) {
+            row = __ldg(idx + j);
+            if (row < 0 || row >= p.m) {
+              record_status(p.status, GRASS_ERR_INVALID_ARG, row);
+              row = -1;
+            }
+          }
+          rows[a][h] = row;
+        }
+      }
+      int tok0 = t.kb_begin * kTcBK;
+      for (int it = 0; it < t.kb_count; ++it) {
+        int ok = 1;
+        if (lane == 0)
+          ok = ptx::mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kTcWaitLimit) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) {
+          if (lane == 0) {
+            if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 400 + s);
+            *abort_flag = 1;
+          }
+          alive = false;
+          break;
+        }
+        uint8_t* stage = tiles + s * STAGE_BYTES + X_SLABS * kTcSlabBytes;
+#pragma unroll
+        for (int a = 0; a < A_SLABS; ++a) {
+          // all loads of this warp's share of the slab first (kTcBK / GW tokens x 2 per lane in
+          // flight), then the stores: the gather is latency-bound otherwise
+          constexpr int NT = kTcBK / GW;
+          unsigned short v0[NT], v1[NT];
+#pragma unroll
+          for (int k = 0; k < NT; ++k) {
+            const int tok = tok0 + g + k * GW;
+            const unsigned short* line = src + static_cast<long long>(tok) * p.lddy;
+            v0[k] = 0;
+            v1[k] = 0;
+            if (tok < p.T) {
+              if (rows[a][0] >= 0) v0[k] = __ldg(line + rows[a][0]);
+              if (rows[a][1] >= 0) v1[k] = __ldg(line + rows[a][1]);
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < NT; ++k) {
+            const int tt = g + k * GW;
+            uint8_t* rowp = stage + a * kTcSlabBytes + tt * 128;
+            const int sw = tt & 7;
+            *reinterpret_cast<unsigned short*>(rowp + (((lane >> 3) ^ sw) << 4) + (lane & 7) * 2) = v0[k];
+            *reinterpret_cast<unsigned short*>(rowp + ((((lane >> 3) + 4) ^ sw) << 4) + (lane & 7) * 2) = v1[k];
+          }
+        }
+        ptx::fence_proxy_async_smem();   // generic writes -> visible to the MMA's async proxy
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive_leader(&bar_full[s]);
+        tok0 += kTcBK;
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
   } else {

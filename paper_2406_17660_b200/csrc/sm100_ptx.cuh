@@ -38,18 +38,40 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
+// The same probe with cluster-scope acquire: for a barrier whose arrivals come from the other
+// CTA of a pair after that CTA wrote shared memory the waiter's MMA is about to read.
+__device__ __forceinline__ bool mbar_test_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Generic-proxy writes to shared memory -> visible to the async proxy (the MMA's operand reads).
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
 // Bounded wait: gives up after `limit_cycles` SM clocks or as soon as *abort is
 // set by another role of this CTA (abort may be NULL).  Returns false on giving up.
 // sleep_ns == 0 spins on test_wait (single-thread pipeline roles: lowest wake-up
 // latency); sleep_ns > 0 backs off between probes (long waits by several warps).
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity,
                                                   volatile int* abort, long long limit_cycles,
-                                                  unsigned sleep_ns = 0) {
-  if (mbar_test_wait(bar, parity)) return true;
+                                                  unsigned sleep_ns = 0,
+                                                  bool cluster_scope = false) {
+  auto probe = [&]() {
+    return cluster_scope ? mbar_test_wait_cluster(bar, parity) : mbar_test_wait(bar, parity);
+  };
+  if (probe()) return true;
   const long long start = clock64();
   unsigned spins = 0;
   while (true) {
-    if (mbar_test_wait(bar, parity)) return true;
+    if (probe()) return true;
     if (sleep_ns != 0) __nanosleep(sleep_ns);
     if ((++spins & 63u) == 0u || sleep_ns != 0) {
       if (abort != nullptr && *abort != 0) return false;
