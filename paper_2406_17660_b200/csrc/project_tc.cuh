@@ -21,6 +21,11 @@
 // tile boundaries; a "TMEM free" barrier returns the accumulators from the epilogue warps to
 // the MMA issuer between tiles.
 //
+// FUSED = true adds eight gather warps that pick the selected dY columns themselves and write
+// them into the B-operand slabs (generic-proxy stores in the swizzled layout, proxy fence,
+// arrive on "full"); the host uses it for small, densely picked tiles, and the gather pre-pass
+// below otherwise.
+//
 // Warp roles (320 threads): warp 0 = TMA producer (one lane per slab), warp 1 =
 // TMEM owner + single-thread MMA issuer, warps 2..9 = epilogue (warp w reads
 // TMEM lanes 32*(w%4)..+31; the two warps of a lane quarter alternate over the
