@@ -125,7 +125,7 @@ __device__ __forceinline__ float warp_transpose_sum(float (&x)[32], int lane) {
 }
 
 template <int MB, int NSLAB, bool PAIR, bool FUSED>
-__global__ void __launch_bounds__(kTcThreads + kTcGatherThreads, 1)
+__global__ void __launch_bounds__(FUSED ? kTcThreads + kTcGatherThreads : kTcThreads, 1)
 project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   constexpr int R_CTA = 64 * NSLAB;          // selected rows per CTA tile (per pair if PAIR)
   constexpr int X_SLABS = 2 * MB;
