@@ -46,10 +46,15 @@ TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false, int gro
   p.MB = 1;
   p.split_k = 1;
   // GRASS_TC_NO_PAIR (diagnostic) keeps every CTA on its own MMA, for A/B timing
-  static const bool no_pair = getenv("GRASS_TC_NO_PAIR") != nullptr;   // read once
+  // diagnostics, read on every call so that a test can sweep them: GRASS_TC_NO_PAIR keeps every
+  // CTA on its own MMA, GRASS_TC_FORCE_MB fixes the n-blocks per CTA (1, 2 or 4, if it fits)
+  const bool no_pair = getenv("GRASS_TC_NO_PAIR") != nullptr;
+  const char* force_mb_env = getenv("GRASS_TC_FORCE_MB");
+  const int force_mb = force_mb_env != nullptr ? atoi(force_mb_env) : 0;
   const bool can_pair = (p.r_cta % 128) == 0 && !no_pair;
   p.pair = false;
   for (int mb = mb_max; mb >= 1; mb /= 2) {
+    if (force_mb > 0 && force_mb <= mb_max && mb != force_mb) continue;
     for (int pair = can_pair ? 1 : 0; pair >= 0; --pair) {
       if (pair && n <= static_cast<int64_t>(mb) * 128) continue;  // nothing for the second CTA
       const int cta_cols = mb * 128 * (pair ? 2 : 1);
@@ -272,9 +277,9 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   // (m = 512, r = 128) step 253 -> 274 TFLOP/s; at m = 2048, r = 128 the sparser pick makes the
   // in-kernel loads the bottleneck (471 -> 379 TFLOP/s), hence the density condition
   // (32 neighbouring picks span 64 / density bytes = 0.5 / density 128-byte lines).
-  static const bool no_fuse = getenv("GRASS_TC_NO_FUSED_GATHER") != nullptr;   // diagnostic
+  const bool no_fuse = getenv("GRASS_TC_NO_FUSED_GATHER") != nullptr;   // diagnostic
   const int tiles_x = plan.pair ? plan.n_blocks / 2 : plan.n_blocks;
-  static const int max_tiles_x = getenv("GRASS_TC_FUSED_MAX_TILES") != nullptr
+  const int max_tiles_x = getenv("GRASS_TC_FUSED_MAX_TILES") != nullptr
                                      ? atoi(getenv("GRASS_TC_FUSED_MAX_TILES")) : 2;   // diagnostic
   const bool fused_gather = gather && !no_fuse && plan.r_cta <= 128 && tiles_x <= max_tiles_x &&
                             static_cast<int64_t>(r) * 12 >= m;  // a 32-lane load then spans <= 6 lines

@@ -259,6 +259,9 @@ def test_project_fp32(T, m, n, r):
     (64, 13824, 256, 13824, None, {"identity": True}),   # largest LLaMA row count, dense: 27 row blocks
     (96, 640, 128, 384, None, {}),                       # 384 rows: MMA chunks of 256 + 128, single CTA
     (96, 640, 512, 384, None, {}),                       # same through a CTA pair
+    (3000, 512, 1024, 128, None, {"dup": True}),         # dense pick, wide n: in-kernel gather
+    (700, 600, 1000, 64, None, {}),                      # in-kernel gather, single CTA, ragged T and n
+    (2100, 256, 2048, 32, None, {}),                     # 32 rows padded to a 64-row tile
 ])
 def test_project_bf16_tensor_core(T, m, n, r, ldx, kw):
     got, want = _project_case(T, m, n, r, torch.bfloat16, seed=T + n + r, ldx=ldx, **kw)
@@ -575,3 +578,25 @@ def test_resume_from_copied_state_is_bit_identical():
     grass.grass_device_status()
     assert torch.equal(a.W, c.W) and torch.equal(a.M, c.M) and torch.equal(a.V, c.V)
     assert torch.equal(a.idx, c.idx)
+
+
+# --------------------------------------------------------------------------- kernel variants
+@pytest.mark.parametrize("force_mb", ["1", "2", "4"])
+@pytest.mark.parametrize("no_pair", [False, True])
+@pytest.mark.parametrize("no_fused", [False, True])
+def test_every_tile_variant_of_the_projection_kernel(force_mb, no_pair, no_fused, monkeypatch):
+    """The host picks the tile shape from a cost model, so a given problem exercises one template
+    instantiation.  The diagnostic switches pin the n-blocks per CTA, single CTAs instead of CTA
+    pairs, and the gather pre-pass instead of the in-kernel gather, so that every instantiation
+    that can serve these shapes is run and checked against the oracle."""
+    monkeypatch.setenv("GRASS_TC_FORCE_MB", force_mb)
+    if no_pair:
+        monkeypatch.setenv("GRASS_TC_NO_PAIR", "1")
+    if no_fused:
+        monkeypatch.setenv("GRASS_TC_NO_FUSED_GATHER", "1")
+    monkeypatch.setenv("GRASS_TC_FUSED_MAX_TILES", "8")
+    for T, m, n, r in [(1500, 512, 1024, 128), (900, 256, 520, 64), (1100, 640, 1024, 256),
+                       (800, 1200, 1024, 448)]:
+        got, want = _project_case(T, m, n, r, torch.bfloat16, seed=T + r, dup=True)
+        err = rel_fro(got, want)
+        assert np.all(np.isfinite(got)) and err <= 1e-4, (T, m, n, r, err)
