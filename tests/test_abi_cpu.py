@@ -57,8 +57,8 @@ def test_argument_errors_are_returned_without_a_device(lib):
                                   null) == 1                                 # ldx < n
     assert lib.grass_project_grad(fake, 8, fake, 12, 1, 16, 8, 8, fake, null, 4, fake, 8, null, 0,
                                   null) == 2                                 # bf16 pitch not 16-byte
-    assert lib.grass_project_grad(fake, 8, fake, 8, 1, 16, 8, 8, fake, null, 4, fake, 8, null, 0,
-                                  null) == 5                                 # bf16 needs workspace
+    assert lib.grass_project_grad(fake, 1000, fake, 8, 1, 16, 1000, 8, fake, null, 4, fake, 8, null,
+                                  0, null) == 5      # sparse pick: the gather pre-pass needs workspace
     assert lib.grass_subspace_adam(fake, 8, fake, fake, fake, 8, 4, 8, 1e-3, 0.9, 0.999, 1e-8, 0,
                                    null) == 1                                # step < 1
     assert lib.grass_subspace_adam(fake, 8, fake, fake, fake, 8, 4, 8, 1e-3, 1.0, 0.999, 1e-8, 1,
