@@ -600,3 +600,33 @@ def test_every_tile_variant_of_the_projection_kernel(force_mb, no_pair, no_fused
         got, want = _project_case(T, m, n, r, torch.bfloat16, seed=T + r, dup=True)
         err = rel_fro(got, want)
         assert np.all(np.isfinite(got)) and err <= 1e-4, (T, m, n, r, err)
+
+
+def test_updates_with_repeated_rows_are_bit_reproducible():
+    """Repeated rows are summed by one owner in a fixed order: two runs give the same bits."""
+    m, n, r = 512, 1376, 256
+    rng = np.random.default_rng(3)
+    sigma = np.sort(rng.choice(40, r, replace=True))          # heavy repetition
+    idx = torch.tensor(sigma, dtype=torch.int32, device=DEV)
+    rho = torch.tensor((0.5 + rng.random(r)).astype(np.float32), device=DEV)
+    g = torch.Generator().manual_seed(1)
+    Gc = torch.randn((r, n), generator=g).to(DEV)
+    W0 = syn.make_W(m, n, torch.bfloat16, seed0=2).to(DEV)
+    outs = []
+    for _ in range(2):
+        W, M, V = W0.clone(), torch.zeros_like(Gc), torch.zeros_like(Gc)
+        grass.grass_adam_scatter(Gc, M, V, None, W, idx, rho, 1e-3, 0.9, 0.999, 1e-8, 1, 0.25)
+        W2 = W0.clone()
+        U = torch.empty_like(Gc)
+        grass.grass_subspace_adam(Gc, torch.zeros_like(Gc), torch.zeros_like(Gc), U, 1e-3, 0.9, 0.999, 1e-8, 1)
+        grass.grass_scatter_update(W2, U, idx, rho, 0.25)
+        grass.grass_device_status()
+        outs.append((W, W2))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    assert torch.equal(outs[0][0], outs[0][1])
+    want = oracle.scatter_update(f64(W0), oracle.adam_update(np.zeros((r, n)), np.zeros((r, n)), f64(Gc),
+                                                            1e-3, 0.9, 0.999, 1e-8, 1)[2],
+                                 sigma, rho.cpu().numpy(), 0.25, w_is_bf16=True)
+    got = f64(outs[0][0])
+    assert np.max(np.abs(got - want)) <= 2.0 ** -7 * np.max(np.abs(want))
+    assert np.mean(got != want) < 0.01
