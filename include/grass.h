@@ -155,7 +155,6 @@ int grass_select_static(const float* norms, int64_t m, int32_t r, int method, ui
  * accepts any alignment.  The sum over tokens is split into a fixed number of
  * slices added in a fixed order: results are bit-reproducible run to run.
  * A row index outside [0, m) contributes zeros and sets the status word.
- * GRASS_BF16 with idx: T <= 2 097 120 tokens (GRASS_ERR_UNSUPPORTED beyond).
  */
 size_t grass_project_workspace_bytes(int64_t T, int64_t m, int64_t n, int32_t r, int dt);
 int grass_project_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx, int dt,
@@ -256,6 +255,63 @@ int grass_adam_scatter_batched(int32_t count, const float* const* Gc, int64_t ld
                                const int32_t* const* idx, const float* const* rho, int32_t r,
                                double lr, double beta1, double beta2, double eps, int32_t step,
                                double alpha, void* stream);
+
+/*
+ * grass_project_grad_batched with the tiling decisions exposed (the paper has no
+ * counterpart: it leaves the product rho ((B dY^T) X) of Section 3.1 to a library
+ * matmul).  By default the library chooses, from (T, m, n, r, count) alone, the
+ * output tile of a CTA, whether two CTAs share each MMA, into how many token slices
+ * the sum over T is split, and how the selected columns of dY reach the tensor
+ * cores.  A grass_project_opts_t (host pointer; NULL = all defaults) overrides any
+ * of these; 0 in a field keeps the default.  Every choice computes the same sums;
+ * results differ only in fp32 summation order (the token slices), and are
+ * bit-reproducible for fixed options.
+ *   gather            GRASS_GATHER_PREPASS: a separate kernel first copies the r
+ *                       selected columns into a token-major T x r matrix in ws
+ *                       (T <= 2 097 120 tokens, GRASS_ERR_UNSUPPORTED beyond).
+ *                     GRASS_GATHER_IN_CTA: every CTA of the GEMM picks the columns
+ *                       of its own tile straight into shared memory (tiles of at
+ *                       most 128 selected rows; otherwise the default is used).
+ *                     GRASS_GATHER_COOPERATIVE: all CTAs of the GEMM share one pass
+ *                       over dY while the MMAs run; the picked columns travel
+ *                       through the T x r matrix in ws, chunk by chunk.
+ *   n_blocks_per_cta  1, 2 or 4 blocks of 128 columns of n per CTA (ignored if the
+ *                     accumulators would not fit).
+ *   cta_pair          GRASS_PAIR_NEVER / GRASS_PAIR_ALWAYS (where r allows it).
+ *   token_slices      number of slices of T (clamped to what T allows).
+ * grass_project_plan reports what a call with these arguments would do, and the
+ * workspace it needs, without touching the GPU (plan: host pointer, written).
+ * grass_project_grad_ex takes the arguments of grass_project_grad_batched plus
+ * opts; ws needs plan->workspace_bytes bytes for the same arguments.
+ */
+enum { GRASS_GATHER_AUTO = 0, GRASS_GATHER_PREPASS = 1, GRASS_GATHER_IN_CTA = 2,
+       GRASS_GATHER_COOPERATIVE = 3 };
+enum { GRASS_PAIR_AUTO = 0, GRASS_PAIR_NEVER = 1, GRASS_PAIR_ALWAYS = 2 };
+typedef struct {
+  int32_t gather;
+  int32_t n_blocks_per_cta;
+  int32_t cta_pair;
+  int32_t token_slices;
+} grass_project_opts_t;
+typedef struct {
+  int32_t gather;            /* GRASS_GATHER_* actually used */
+  int32_t rows_per_tile;     /* selected rows per CTA tile (a multiple of 64) */
+  int32_t row_blocks;        /* tiles along r */
+  int32_t n_blocks_per_cta;
+  int32_t ctas_per_slice;    /* CTAs that share one token slice, over all `count` layers */
+  int32_t cta_pair;          /* 1: two CTAs per MMA */
+  int32_t token_slices;
+  int32_t tokens_per_stage;  /* tokens per pipeline stage (32 or 64) */
+  int32_t stages;
+  size_t workspace_bytes;
+} grass_project_plan_t;
+int grass_project_plan(int32_t count, int64_t T, int64_t m, int64_t n, int32_t r,
+                       const grass_project_opts_t* opts, grass_project_plan_t* plan);
+int grass_project_grad_ex(int32_t count, const void* const* dY, int64_t lddy,
+                          const void* const* X, int64_t ldx, int64_t T, int64_t m, int64_t n,
+                          const int32_t* const* idx, const float* const* rho, int32_t r,
+                          float* const* Gc, int64_t ldgc, void* ws, size_t ws_bytes,
+                          const grass_project_opts_t* opts, void* stream);
 
 /*
  * Column form of the apply step, for layers projected on their input dimension

@@ -12,7 +12,9 @@ from .binding import (  # noqa: F401
     grass_project_grad, grass_project_workspace_bytes,
     grass_grad_row_norms, grass_grad_row_norms_workspace_bytes,
     grass_subspace_adam, grass_adam_scatter, grass_adam_scatter_batched,
-    grass_project_grad_batched, grass_project_batched_workspace_bytes, grass_scatter_update, grass_scatter_update_cols, grass_device_status,
+    grass_project_grad_batched, grass_project_batched_workspace_bytes,
+    grass_project_grad_ex, grass_project_plan, ProjectOpts, GATHER_AUTO, GATHER_PREPASS, GATHER_IN_CTA,
+    GATHER_COOPERATIVE, PAIR_AUTO, PAIR_NEVER, PAIR_ALWAYS, grass_scatter_update, grass_scatter_update_cols, grass_device_status,
     grass_status_string, grass_profile_begin, grass_profile_end, grass_profile_end_timeline, grass_selftest_bounded_wait, library_path, load_library,
 )
 from .step import GrassLayer  # noqa: F401

@@ -306,6 +306,63 @@ _SIGNATURES_BATCHED = {
 }
 _SIGNATURES.update(_SIGNATURES_BATCHED)
 
+GATHER_AUTO, GATHER_PREPASS, GATHER_IN_CTA, GATHER_COOPERATIVE = 0, 1, 2, 3
+PAIR_AUTO, PAIR_NEVER, PAIR_ALWAYS = 0, 1, 2
+
+
+class ProjectOpts(ctypes.Structure):
+    """grass_project_opts_t: 0 in a field keeps the library's own choice."""
+    _fields_ = [("gather", c_int32), ("n_blocks_per_cta", c_int32), ("cta_pair", c_int32),
+                ("token_slices", c_int32)]
+
+
+class ProjectPlan(ctypes.Structure):
+    """grass_project_plan_t."""
+    _fields_ = [("gather", c_int32), ("rows_per_tile", c_int32), ("row_blocks", c_int32),
+                ("n_blocks_per_cta", c_int32), ("ctas_per_slice", c_int32), ("cta_pair", c_int32),
+                ("token_slices", c_int32), ("tokens_per_stage", c_int32), ("stages", c_int32),
+                ("workspace_bytes", c_size_t)]
+
+
+_SIGNATURES.update({
+    "grass_project_plan": (c_int, [c_int32, c_int64, c_int64, c_int64, c_int32,
+                                   ctypes.POINTER(ProjectOpts), ctypes.POINTER(ProjectPlan)]),
+    "grass_project_grad_ex": (c_int, [c_int32, c_void_p, c_int64, c_void_p, c_int64, c_int64, c_int64,
+                                      c_int64, c_void_p, c_void_p, c_int32, c_void_p, c_int64,
+                                      c_void_p, c_size_t, ctypes.POINTER(ProjectOpts), c_void_p]),
+})
+
+
+def _opts(opts):
+    if opts is None:
+        return None
+    if isinstance(opts, ProjectOpts):
+        return ctypes.byref(opts)
+    return ctypes.byref(ProjectOpts(**opts))
+
+
+def grass_project_plan(count: int, T: int, m: int, n: int, r: int, opts=None) -> dict:
+    """What grass_project_grad_ex would do for these arguments (host only, no GPU needed)."""
+    plan = ProjectPlan()
+    _check(load_library().grass_project_plan(count, T, m, n, r, _opts(opts), ctypes.byref(plan)),
+           "grass_project_plan")
+    return {name: int(getattr(plan, name)) for name, _ in ProjectPlan._fields_}
+
+
+def grass_project_grad_ex(dYs, Xs, idxs, rhos, r, Gcs, ws, opts=None) -> None:
+    count = len(dYs)
+    T, m = dYs[0].shape
+    n = Xs[0].shape[1]
+    for t in Gcs:
+        _require(t, torch.float32, "Gc")
+    for t in idxs:
+        _require(t, torch.int32, "idx")
+    keep = (_ptr_array(dYs), _ptr_array(Xs), _ptr_array(idxs), _ptr_array(rhos), _ptr_array(Gcs))
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(load_library().grass_project_grad_ex(
+        count, keep[0], _ld(dYs[0]), keep[1], _ld(Xs[0]), T, m, n, keep[2], keep[3], r, keep[4],
+        _ld(Gcs[0]), _ptr(ws), ws_bytes, _opts(opts), _stream()), "grass_project_grad_ex")
+
 
 def _ptr_array(tensors):
     """Host array of device pointers (None entries become NULL); None -> NULL array."""

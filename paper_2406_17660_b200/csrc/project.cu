@@ -2,7 +2,6 @@
 // launches).  The kernels are in project_tc.cuh (bf16, tcgen05) and
 // project_simt.cuh (fp32).
 #include <cudaTypedefs.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 #include "project_simt.cuh"
@@ -13,7 +12,39 @@ namespace {
 
 constexpr int kSmCount = 148;
 
+// How the selected dY columns reach the GEMM (values of grass_project_opts_t::gather; 0 in a
+// plan means the operand is dY itself, i.e. the dense gradient).
+constexpr int kOptAuto = 0, kOptPrepass = 1, kOptCta = 2, kOptCoop = 3;
+
+struct PlanOpts {
+  int gather = kOptAuto;   // kOpt*
+  int mb = 0;              // n-blocks of 128 columns per CTA: 0 = cost model, else 1, 2 or 4 if it fits
+  int pair = 0;            // 0 = cost model, 1 = single CTAs only, 2 = CTA pairs wherever the shape allows
+  int split = 0;           // token slices: 0 = cost model
+};
+
+PlanOpts to_plan_opts(const grass_project_opts_t* o) {
+  PlanOpts po;
+  if (o != nullptr) {
+    po.gather = o->gather;
+    po.mb = o->n_blocks_per_cta;
+    po.pair = o->cta_pair;
+    po.split = o->token_slices;
+  }
+  return po;
+}
+bool opts_ok(const grass_project_opts_t* o) {
+  return o == nullptr ||
+         (o->gather >= kOptAuto && o->gather <= kOptCoop &&
+          (o->n_blocks_per_cta == 0 || o->n_blocks_per_cta == 1 || o->n_blocks_per_cta == 2 ||
+           o->n_blocks_per_cta == 4) &&
+          o->cta_pair >= 0 && o->cta_pair <= 2 && o->token_slices >= 0);
+}
+
 struct TcPlan {
+  int gather;     // 0: operand read from dY as it is; else kOptPrepass / kOptCta / kOptCoop
+  int kb_unit;    // token slices start on multiples of this many token blocks
+  size_t ctrl_bytes;   // cooperative gather: queue head and per-chunk counters
   int r_pad;      // r_blocks * r_cta: width of the gathered operand
   int r_cta, r_blocks;
   int MB, n_blocks;   // n_blocks = gridDim.x (CTAs, an even number when pair)
@@ -30,7 +61,8 @@ struct TcPlan {
 // n-tiles (MB) make more, smaller CTAs, which cuts partial traffic when the
 // output is tiny; larger ones cut the number of times the gathered operand is
 // re-read.  The result depends only on (T, n, r), so it is reproducible.
-TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false, int groups = 1) {
+TcPlan make_plan(int64_t T, int64_t m, int64_t n, int r, bool has_idx, const PlanOpts& opts,
+                 bool single_split = false, int groups = 1) {
   TcPlan p;
   const int r64 = static_cast<int>(round_up(static_cast<size_t>(r), 64));
   p.r_blocks = (r64 + 511) / 512;
@@ -45,18 +77,14 @@ TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false, int gro
   double best = 1e300;
   p.MB = 1;
   p.split_k = 1;
-  // GRASS_TC_NO_PAIR (diagnostic) keeps every CTA on its own MMA, for A/B timing
-  // diagnostics, read on every call so that a test can sweep them: GRASS_TC_NO_PAIR keeps every
-  // CTA on its own MMA, GRASS_TC_FORCE_MB fixes the n-blocks per CTA (1, 2 or 4, if it fits)
-  const bool no_pair = getenv("GRASS_TC_NO_PAIR") != nullptr;
-  const char* force_mb_env = getenv("GRASS_TC_FORCE_MB");
-  const int force_mb = force_mb_env != nullptr ? atoi(force_mb_env) : 0;
-  const bool can_pair = (p.r_cta % 128) == 0 && !no_pair;
+  const int force_mb = opts.mb;
+  const bool can_pair = (p.r_cta % 128) == 0 && opts.pair != 1;
   p.pair = false;
   for (int mb = mb_max; mb >= 1; mb /= 2) {
     if (force_mb > 0 && force_mb <= mb_max && mb != force_mb) continue;
     for (int pair = can_pair ? 1 : 0; pair >= 0; --pair) {
       if (pair && n <= static_cast<int64_t>(mb) * 128) continue;  // nothing for the second CTA
+      if (!pair && opts.pair == 2 && can_pair && n > static_cast<int64_t>(mb) * 128) continue;
       const int cta_cols = mb * 128 * (pair ? 2 : 1);
       const int n_tiles = static_cast<int>((n + cta_cols - 1) / cta_cols);
       const int64_t tiles =
@@ -68,6 +96,7 @@ TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false, int gro
       const double fixed = 3000.0 + mb * 128.0 * p.r_cta * 4.0 / 128.0;
       const int max_s = single_split ? 1 : (p.k_blocks < 256 ? p.k_blocks : 256);
       for (int s = 1; s <= max_s; ++s) {
+        if (opts.split > 0 && !single_split && s != (opts.split < max_s ? opts.split : max_s)) continue;
         const int64_t ctas = tiles * s;
         const int64_t waves = (ctas + kSmCount - 1) / kSmCount;
         const double blocks_per_cta = static_cast<double>((p.k_blocks + s - 1) / s);
@@ -89,11 +118,40 @@ TcPlan make_plan(int64_t T, int64_t n, int r, bool single_split = false, int gro
   const int a_slabs = p.pair ? p.r_cta / 128 : p.r_cta / 64;
   p.bk = tc_bk(p.MB, a_slabs);
   p.k_blocks = static_cast<int>((T + p.bk - 1) / p.bk);
-  if (p.split_k > p.k_blocks) p.split_k = p.k_blocks;
+  // How the selected columns get to the GEMM.  In-CTA gather: the GEMM's own warps pick the
+  // columns out of dY into shared memory.  It pays when a tile holds at most 128 rows (the load
+  // unit keeps up), at most two CTAs (pairs) share a token slice (each gathers for itself) and
+  // the picks are dense enough that a 32-lane load spans at most 6 cache lines (12 r >= m);
+  // measured on the 60M q,k,v,o group (m = 512, r = 128): step 253 -> 274 TFLOP/s, while at
+  // m = 2048, r = 128 the sparser pick made the in-kernel loads the bottleneck (471 -> 379).
+  // Everything else: cooperative gather (all CTAs share one pass over dY, overlapped with the
+  // MMAs); the stand-alone pre-pass remains selectable.
+  p.gather = 0;
+  if (has_idx) {
+    const int tiles_x = p.pair ? p.n_blocks / 2 : p.n_blocks;
+    const bool cta_ok = p.r_cta <= 128;
+    if (opts.gather == kOptCta && cta_ok) p.gather = kOptCta;
+    else if (opts.gather == kOptPrepass) p.gather = kOptPrepass;
+    else if (opts.gather == kOptCoop) p.gather = kOptCoop;
+    else if (opts.gather == kOptAuto && cta_ok && tiles_x <= 2 && static_cast<int64_t>(r) * 12 >= m)
+      p.gather = kOptCta;
+    else p.gather = kOptCoop;
+  }
+  p.kb_unit = p.gather == kOptCoop ? kCoopChunk / p.bk : 1;
+  {
+    const int n_units = (p.k_blocks + p.kb_unit - 1) / p.kb_unit;
+    if (p.split_k > n_units) p.split_k = n_units;
+  }
+  p.ctrl_bytes = p.gather == kOptCoop
+                     ? round_up((kCoopCtrlInts + static_cast<size_t>(groups) *
+                                                     ((T + kCoopChunk - 1) / kCoopChunk)) * sizeof(int), 256)
+                     : 0;
   p.stages = tc_stages(p.MB, a_slabs);
   p.smem_bytes = static_cast<size_t>(p.stages) * tc_stage_bytes(p.MB, a_slabs) + 1024;
   p.ld_part = static_cast<long long>(round_up(static_cast<size_t>(n), 4));
-  p.ag_bytes = round_up(static_cast<size_t>(T) * p.r_pad * sizeof(__nv_bfloat16), 256);
+  p.ag_bytes = p.gather == kOptPrepass || p.gather == kOptCoop
+                   ? round_up(static_cast<size_t>(T) * p.r_pad * sizeof(__nv_bfloat16), 256)
+                   : 0;
   p.part_bytes = p.split_k > 1
                      ? round_up(static_cast<size_t>(p.split_k) * r * p.ld_part * sizeof(float), 256)
                      : 0;
@@ -130,8 +188,9 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
   return true;
 }
 
-template <int MB, int NSLAB, bool PAIR, bool FUSED>
+template <int MB, int NSLAB, bool PAIR, int GATHER>
 int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& maps, TcParams p) {
+  constexpr bool FUSED = GATHER != kGatherNone;   // the variants with eight extra warps
   static bool attr_set[64] = {false};
   static int max_workers[64] = {0};
   int dev = 0;
@@ -149,14 +208,14 @@ int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& map
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (!attr_set[dev]) {
-    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel<MB, NSLAB, PAIR, FUSED>,
+    GRASS_CUDA_TRY(cudaFuncSetAttribute(project_tc_kernel<MB, NSLAB, PAIR, GATHER>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kTcSmemBudget));
     // how many workers (CTAs, or CTA pairs) the device holds at once: one per SM / SM pair
     int workers = 0;
     if (PAIR) {
       cfg.gridDim = dim3(2 * kSmCount);
-      GRASS_CUDA_TRY(cudaOccupancyMaxActiveClusters(&workers, project_tc_kernel<MB, NSLAB, PAIR, FUSED>,
+      GRASS_CUDA_TRY(cudaOccupancyMaxActiveClusters(&workers, project_tc_kernel<MB, NSLAB, PAIR, GATHER>,
                                                     &cfg));
     } else {
       GRASS_CUDA_TRY(cudaDeviceGetAttribute(&workers, cudaDevAttrMultiProcessorCount, dev));
@@ -170,40 +229,44 @@ int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& map
   p.tiles_y = static_cast<int>(tile_grid.y);
   p.tiles_z = static_cast<int>(tile_grid.z);
   const long long n_tiles = static_cast<long long>(tile_grid.x) * tile_grid.y * tile_grid.z;
-  const int workers = n_tiles < max_workers[dev] ? static_cast<int>(n_tiles) : max_workers[dev];
+  // (cooperative gather: every SM takes part in the gather, also those without a tile)
+  const int workers = n_tiles < max_workers[dev] && GATHER != kGatherCoop ? static_cast<int>(n_tiles)
+                                                                          : max_workers[dev];
   cfg.gridDim = dim3(static_cast<unsigned>(PAIR ? 2 * workers : workers));
   {
     ProfileScope prof(GRASS_K_PROJECT_TC, s);
-    GRASS_CUDA_TRY(cudaLaunchKernelEx(&cfg, project_tc_kernel<MB, NSLAB, PAIR, FUSED>, maps, p));
+    GRASS_CUDA_TRY(cudaLaunchKernelEx(&cfg, project_tc_kernel<MB, NSLAB, PAIR, GATHER>, maps, p));
   }
   return GRASS_OK;
 }
 
 // (MB, NSLAB) with MB * 64 * NSLAB <= 512 TMEM columns; pairs need an even NSLAB.
-int launch_tc(int MB, int nslab, bool pair, bool fused, dim3 grid, size_t smem, cudaStream_t s,
+// gather: kGatherNone / kGatherCta (tiles of at most 128 rows) / kGatherCoop.
+int launch_tc(int MB, int nslab, bool pair, int gather, dim3 grid, size_t smem, cudaStream_t s,
               const TcMaps& maps, const TcParams& p) {
-#define GRASS_TC_CASE(mb, ns)                                                                  \
-  if (MB == mb && nslab == ns && !pair && !fused)                                              \
-    return launch_tc_one<mb, ns, false, false>(grid, smem, s, maps, p)
-#define GRASS_TC_PAIR(mb, ns)                                                                  \
-  if (MB == mb && nslab == ns && pair && !fused)                                               \
-    return launch_tc_one<mb, ns, true, false>(grid, smem, s, maps, p)
-#define GRASS_TC_FUSED(mb, ns, pr)                                                             \
-  if (MB == mb && nslab == ns && pair == pr && fused)                                          \
-    return launch_tc_one<mb, ns, pr, true>(grid, smem, s, maps, p)
-  GRASS_TC_CASE(1, 1); GRASS_TC_CASE(1, 2); GRASS_TC_CASE(1, 3); GRASS_TC_CASE(1, 4);
-  GRASS_TC_CASE(1, 5); GRASS_TC_CASE(1, 6); GRASS_TC_CASE(1, 7); GRASS_TC_CASE(1, 8);
-  GRASS_TC_CASE(2, 1); GRASS_TC_CASE(2, 2); GRASS_TC_CASE(2, 3); GRASS_TC_CASE(2, 4);
-  GRASS_TC_CASE(4, 1); GRASS_TC_CASE(4, 2);
-  GRASS_TC_PAIR(1, 2); GRASS_TC_PAIR(1, 4); GRASS_TC_PAIR(1, 6); GRASS_TC_PAIR(1, 8);
-  GRASS_TC_PAIR(2, 2); GRASS_TC_PAIR(2, 4); GRASS_TC_PAIR(4, 2);
-  // in-kernel gather: at most 128 selected rows per tile
-  GRASS_TC_FUSED(1, 1, false); GRASS_TC_FUSED(2, 1, false); GRASS_TC_FUSED(4, 1, false);
-  GRASS_TC_FUSED(1, 2, false); GRASS_TC_FUSED(2, 2, false); GRASS_TC_FUSED(4, 2, false);
-  GRASS_TC_FUSED(1, 2, true); GRASS_TC_FUSED(2, 2, true); GRASS_TC_FUSED(4, 2, true);
-#undef GRASS_TC_FUSED
+#define GRASS_TC_CASE(mb, ns, pr, ga)                                                          \
+  if (MB == mb && nslab == ns && pair == pr && gather == ga)                                   \
+    return launch_tc_one<mb, ns, pr, ga>(grid, smem, s, maps, p)
+#define GRASS_TC_BOTH(mb, ns, pr)                                                              \
+  GRASS_TC_CASE(mb, ns, pr, kGatherNone);                                                      \
+  GRASS_TC_CASE(mb, ns, pr, kGatherCoop)
+  GRASS_TC_BOTH(1, 1, false); GRASS_TC_BOTH(1, 2, false); GRASS_TC_BOTH(1, 3, false);
+  GRASS_TC_BOTH(1, 4, false); GRASS_TC_BOTH(1, 5, false); GRASS_TC_BOTH(1, 6, false);
+  GRASS_TC_BOTH(1, 7, false); GRASS_TC_BOTH(1, 8, false);
+  GRASS_TC_BOTH(2, 1, false); GRASS_TC_BOTH(2, 2, false); GRASS_TC_BOTH(2, 3, false);
+  GRASS_TC_BOTH(2, 4, false);
+  GRASS_TC_BOTH(4, 1, false); GRASS_TC_BOTH(4, 2, false);
+  GRASS_TC_BOTH(1, 2, true); GRASS_TC_BOTH(1, 4, true); GRASS_TC_BOTH(1, 6, true);
+  GRASS_TC_BOTH(1, 8, true);
+  GRASS_TC_BOTH(2, 2, true); GRASS_TC_BOTH(2, 4, true); GRASS_TC_BOTH(4, 2, true);
+  // in-CTA gather: at most 128 selected rows per tile
+  GRASS_TC_CASE(1, 1, false, kGatherCta); GRASS_TC_CASE(2, 1, false, kGatherCta);
+  GRASS_TC_CASE(4, 1, false, kGatherCta); GRASS_TC_CASE(1, 2, false, kGatherCta);
+  GRASS_TC_CASE(2, 2, false, kGatherCta); GRASS_TC_CASE(4, 2, false, kGatherCta);
+  GRASS_TC_CASE(1, 2, true, kGatherCta); GRASS_TC_CASE(2, 2, true, kGatherCta);
+  GRASS_TC_CASE(4, 2, true, kGatherCta);
+#undef GRASS_TC_BOTH
 #undef GRASS_TC_CASE
-#undef GRASS_TC_PAIR
   return GRASS_ERR_UNSUPPORTED;
 }
 
@@ -243,24 +306,29 @@ Fp32Plan make_fp32_plan(int64_t T, int64_t n, int r) {
 // to occupy the GPU (every LLaMA shape from 1B up).  A small gradient (few tiles) would leave
 // most SMs idle, so it is computed with the usual token split into fp32 partials -- small by
 // the same token -- and splitk_rownorms_kernel sums, squares and reduces them.
-TcPlan make_norms_plan(int64_t T, int64_t n, int r) {
-  const TcPlan fused = make_plan(T, n, r, true);
+TcPlan make_norms_plan(int64_t T, int64_t m, int64_t n) {
+  const PlanOpts none;
+  const TcPlan fused = make_plan(T, m, n, static_cast<int>(m), false, none, true);
   if (static_cast<int64_t>(fused.n_blocks) * fused.r_blocks >= 120) return fused;
-  return make_plan(T, n, r, false);
+  return make_plan(T, m, n, static_cast<int>(m), false, none, false);
+}
+
+// Bytes of workspace a plan needs for `count` layers: [control block][per layer: gathered operand,
+// split-K partials].
+size_t plan_ws_bytes(const TcPlan& plan, int count) {
+  return plan.ctrl_bytes + (plan.ag_bytes + plan.part_bytes) * static_cast<size_t>(count);
 }
 
 // Projection of `count` same-shaped layers in one set of launches (count = 1 for the plain
 // call).  norms != NULL (count must be 1): row-norm mode (idx NULL, r == m): the GEMM's epilogue
 // reduces squares instead of storing the gradient, then the partial sums are finalised.
-// Workspace layout: per layer [gathered operand][split-K partials], layers back to back.
 int project_bf16(int count, const void* const* dY, int64_t lddy, const void* const* X, int64_t ldx,
                  int64_t T, int64_t m, int64_t n, const int32_t* const* idx,
                  const float* const* rho, int r, float* const* Gc, int64_t ldgc, float* norms,
-                 void* ws, size_t ws_bytes, cudaStream_t s) {
+                 void* ws, size_t ws_bytes, const PlanOpts& opts, cudaStream_t s) {
   if (count < 1 || count > kTcMaxGroup || (norms != nullptr && count != 1))
     return GRASS_ERR_INVALID_ARG;
   const bool gather = idx != nullptr && idx[0] != nullptr;
-  if (gather && T > 65535LL * kGatherTokens) return GRASS_ERR_UNSUPPORTED;   // gather grid.y
   for (int g = 0; g < count; ++g) {
     if (dY[g] == nullptr || X[g] == nullptr || (norms == nullptr && Gc[g] == nullptr))
       return GRASS_ERR_INVALID_ARG;
@@ -268,24 +336,13 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
     if (!aligned_to(X[g], 16) || ldx % 8 != 0) return GRASS_ERR_ALIGNMENT;
     if (!gather && (!aligned_to(dY[g], 16) || lddy % 8 != 0)) return GRASS_ERR_ALIGNMENT;
   }
-  const TcPlan plan = norms != nullptr ? make_norms_plan(T, n, r) : make_plan(T, n, r, false, count);
+  const TcPlan plan = norms != nullptr ? make_norms_plan(T, m, n)
+                                       : make_plan(T, m, n, r, gather, opts, false, count);
+  if (plan.gather == kOptPrepass && T > 65535LL * kGatherTokens)
+    return GRASS_ERR_UNSUPPORTED;                                            // pre-pass grid.y
   const bool fused_norms = norms != nullptr && plan.split_k == 1;
-  // In-kernel gather: the GEMM's own warps pick the selected columns out of dY.  It pays when a
-  // tile holds at most 128 rows (the load unit keeps up) and at most two CTAs (pairs) share a
-  // token slice (each of them gathers for itself): then the copy pre-pass, its launch and the
-  // round trip of the gathered operand through HBM all disappear.  Measured: 60M q,k,v,o group
-  // (m = 512, r = 128) step 253 -> 274 TFLOP/s; at m = 2048, r = 128 the sparser pick makes the
-  // in-kernel loads the bottleneck (471 -> 379 TFLOP/s), hence the density condition
-  // (32 neighbouring picks span 64 / density bytes = 0.5 / density 128-byte lines).
-  const bool no_fuse = getenv("GRASS_TC_NO_FUSED_GATHER") != nullptr;   // diagnostic
-  const int tiles_x = plan.pair ? plan.n_blocks / 2 : plan.n_blocks;
-  const int max_tiles_x = getenv("GRASS_TC_FUSED_MAX_TILES") != nullptr
-                                     ? atoi(getenv("GRASS_TC_FUSED_MAX_TILES")) : 2;   // diagnostic
-  const bool fused_gather = gather && !no_fuse && plan.r_cta <= 128 && tiles_x <= max_tiles_x &&
-                            static_cast<int64_t>(r) * 12 >= m;  // a 32-lane load then spans <= 6 lines
-  const size_t per_layer = fused_norms ? norm_part_bytes(m, n)
-                                       : (gather && !fused_gather ? plan.ag_bytes : 0) + plan.part_bytes;
-  const size_t need = per_layer * count;
+  const size_t per_layer = fused_norms ? norm_part_bytes(m, n) : plan.ag_bytes + plan.part_bytes;
+  const size_t need = plan.ctrl_bytes + per_layer * count;
   if (need > 0 && (ws == nullptr || !aligned_to(ws, 256) || ws_bytes < need))
     return GRASS_ERR_WORKSPACE;
   cudaError_t err;
@@ -295,17 +352,16 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   TcMaps maps;
   GatherGroup gg;
   float* part[kTcMaxGroup];
+  char* const layers_ws = static_cast<char*>(ws) + plan.ctrl_bytes;
   for (int g = 0; g < count; ++g) {
-    char* wsp = static_cast<char*>(ws) + per_layer * g;
+    char* wsp = layers_ws + per_layer * g;
     if (!make_map(&maps.x[g], X[g], T, n, ldx, plan.bk)) return GRASS_ERR_CUDA;
-    if (fused_gather) {
-      gg.dY[g] = static_cast<const __nv_bfloat16*>(dY[g]);
-      gg.idx[g] = idx[g];
-      gg.Ag[g] = nullptr;
+    gg.dY[g] = static_cast<const __nv_bfloat16*>(dY[g]);
+    gg.idx[g] = gather ? idx[g] : nullptr;
+    gg.Ag[g] = nullptr;
+    if (plan.gather == kOptCta) {
       maps.a[g] = maps.x[g];          // unused by the kernel
-    } else if (gather) {
-      gg.dY[g] = static_cast<const __nv_bfloat16*>(dY[g]);
-      gg.idx[g] = idx[g];
+    } else if (plan.gather == kOptPrepass || plan.gather == kOptCoop) {
       gg.Ag[g] = reinterpret_cast<__nv_bfloat16*>(wsp);
       if (!make_map(&maps.a[g], gg.Ag[g], T, plan.r_pad, plan.r_pad, plan.bk)) return GRASS_ERR_CUDA;
       wsp += plan.ag_bytes;
@@ -319,7 +375,7 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
     maps.a[g] = maps.a[0];
     gg.dY[g] = nullptr; gg.idx[g] = nullptr; gg.Ag[g] = nullptr;
   }
-  if (gather && !fused_gather) {
+  if (plan.gather == kOptPrepass) {
     ProfileScope prof(GRASS_K_GATHER, s);
     const int ni = plan.r_pad >= 256 ? 8 : plan.r_pad / 32;   // r_pad is a multiple of 64
     dim3 ggrid(static_cast<unsigned>((plan.r_pad + 32 * ni - 1) / (32 * ni)),
@@ -337,22 +393,32 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   p.r = r;
   p.k_blocks = plan.k_blocks;
   p.split_k = plan.split_k;
+  p.kb_unit = plan.kb_unit;
   p.status = status;
   p.norm_part = fused_norms ? part[0] : nullptr;
+  const bool in_kernel = plan.gather == kOptCta || plan.gather == kOptCoop;
   for (int g = 0; g < kTcMaxGroup; ++g) {
     const int gi = g < count ? g : 0;
-    p.dY[g] = fused_gather ? gg.dY[gi] : nullptr;
-    p.idx[g] = fused_gather ? gg.idx[gi] : nullptr;
+    p.dY[g] = in_kernel ? gg.dY[gi] : nullptr;
+    p.idx[g] = in_kernel ? gg.idx[gi] : nullptr;
+    p.Ag[g] = plan.gather == kOptCoop ? gg.Ag[gi] : nullptr;
   }
   p.lddy = lddy;
   p.m = static_cast<int>(m);
+  p.r_pad = plan.r_pad;
+  p.coop_ctrl = nullptr;
+  p.coop_chunks = static_cast<int>((T + kCoopChunk - 1) / kCoopChunk);
+  p.coop_cg = (plan.r_pad + kCoopCols - 1) / kCoopCols;
+  {
+    const int n_units = (plan.k_blocks + plan.kb_unit - 1) / plan.kb_unit;
+    p.coop_pmax = n_units / plan.split_k + (n_units % plan.split_k != 0 ? 1 : 0);
+  }
+  if (plan.gather == kOptCoop) {
+    // queue head and per-chunk counters start at zero for every launch
+    p.coop_ctrl = static_cast<int*>(ws);
+    GRASS_CUDA_TRY(cudaMemsetAsync(ws, 0, plan.ctrl_bytes, s));
+  }
   p.ld_norm = static_cast<long long>(round_up(static_cast<size_t>(m), 32));
-  static const bool debug_plan = getenv("GRASS_DEBUG_PLAN") != nullptr;   // read once
-  if (debug_plan)
-    fprintf(stderr, "grass plan T=%lld n=%lld r=%d x%d: r_cta=%d r_blocks=%d MB=%d n_blocks=%d "
-                    "split_k=%d stages=%d pair=%d fused_gather=%d\n", static_cast<long long>(T),
-            static_cast<long long>(n), r, count, plan.r_cta, plan.r_blocks, plan.MB, plan.n_blocks,
-            plan.split_k, plan.stages, plan.pair ? 1 : 0, fused_gather ? 1 : 0);
   for (int g = 0; g < kTcMaxGroup; ++g) {
     const int gi = g < count ? g : 0;
     if (plan.split_k == 1) {
@@ -368,7 +434,10 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   // tile space handed to the persistent kernel (x counts pairs of CTAs in pair mode)
   dim3 grid(static_cast<unsigned>(plan.pair ? plan.n_blocks / 2 : plan.n_blocks),
             static_cast<unsigned>(plan.r_blocks), static_cast<unsigned>(plan.split_k * count));
-  const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, fused_gather, grid, plan.smem_bytes, s, maps, p);
+  const int kernel_gather = plan.gather == kOptCta ? kGatherCta
+                            : plan.gather == kOptCoop ? kGatherCoop : kGatherNone;
+  const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, kernel_gather, grid, plan.smem_bytes,
+                           s, maps, p);
   if (rc != GRASS_OK) return rc;
   if (norms != nullptr) {
     ProfileScope prof(GRASS_K_ROW_NORMS, s);
@@ -404,34 +473,37 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   return GRASS_OK;
 }
 
+void describe_plan(const TcPlan& plan, int count, grass_project_plan_t* out) {
+  out->gather = plan.gather;
+  out->rows_per_tile = plan.r_cta;
+  out->row_blocks = plan.r_blocks;
+  out->n_blocks_per_cta = plan.MB;
+  out->ctas_per_slice = plan.n_blocks * plan.r_blocks * count;
+  out->cta_pair = plan.pair ? 1 : 0;
+  out->token_slices = plan.split_k;
+  out->tokens_per_stage = plan.bk;
+  out->stages = plan.stages;
+  out->workspace_bytes = plan_ws_bytes(plan, count) + 256;
+}
+
 }  // namespace
 }  // namespace grass
 
 extern "C" size_t grass_project_workspace_bytes(int64_t T, int64_t m, int64_t n, int32_t r,
                                                 int dt) {
-  (void)m;
-  if (T < 1 || n < 1 || r < 1) return 0;
+  if (T < 1 || m < 1 || n < 1 || r < 1) return 0;
   if (dt != GRASS_BF16) return grass::make_fp32_plan(T, n, r).part_bytes + 256;
-  const grass::TcPlan plan = grass::make_plan(T, n, r);
-  return plan.ag_bytes + plan.part_bytes + 256;
+  // covers the call with and without idx (the dense form needs no gathered operand)
+  const size_t with_idx = grass::plan_ws_bytes(grass::make_plan(T, m, n, r, true, grass::PlanOpts()), 1);
+  const size_t dense = grass::plan_ws_bytes(grass::make_plan(T, m, n, r, false, grass::PlanOpts()), 1);
+  return (with_idx > dense ? with_idx : dense) + 256;
 }
 
-extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx, int dt,
-                                  int64_t T, int64_t m, int64_t n, const int32_t* idx,
-                                  const float* rho, int32_t r, float* Gc, int64_t ldgc, void* ws,
-                                  size_t ws_bytes, void* stream) {
-  using namespace grass;
-  if (dY == nullptr || X == nullptr || Gc == nullptr || T < 1 || m < 1 || n < 1 || r < 1 ||
-      lddy < m || ldx < n || ldgc < n || T > 0x7fffffffLL || m > 0x7fffffffLL ||
-      n > 0x7fffffffLL)
-    return GRASS_ERR_INVALID_ARG;
-  if (idx == nullptr && r != m) return GRASS_ERR_INVALID_ARG;
-  if (r > m) return GRASS_ERR_INVALID_ARG;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (dt == GRASS_BF16)
-    return project_bf16(1, &dY, lddy, &X, ldx, T, m, n, idx != nullptr ? &idx : nullptr, &rho, r,
-                        &Gc, ldgc, nullptr, ws, ws_bytes, s);
-  if (dt != GRASS_F32) return GRASS_ERR_UNSUPPORTED;
+namespace grass {
+namespace {
+int project_fp32(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T, int64_t m,
+                 int64_t n, const int32_t* idx, const float* rho, int32_t r, float* Gc,
+                 int64_t ldgc, void* ws, size_t ws_bytes, cudaStream_t s) {
   cudaError_t err;
   int* status = status_word(&err);
   if (status == nullptr) GRASS_CUDA_TRY(err);
@@ -464,13 +536,33 @@ extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, i
   }
   return GRASS_OK;
 }
+}  // namespace
+}  // namespace grass
+
+extern "C" int grass_project_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx, int dt,
+                                  int64_t T, int64_t m, int64_t n, const int32_t* idx,
+                                  const float* rho, int32_t r, float* Gc, int64_t ldgc, void* ws,
+                                  size_t ws_bytes, void* stream) {
+  using namespace grass;
+  if (dY == nullptr || X == nullptr || Gc == nullptr || T < 1 || m < 1 || n < 1 || r < 1 ||
+      lddy < m || ldx < n || ldgc < n || T > 0x7fffffffLL || m > 0x7fffffffLL ||
+      n > 0x7fffffffLL)
+    return GRASS_ERR_INVALID_ARG;
+  if (idx == nullptr && r != m) return GRASS_ERR_INVALID_ARG;
+  if (r > m) return GRASS_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dt == GRASS_BF16)
+    return project_bf16(1, &dY, lddy, &X, ldx, T, m, n, idx != nullptr ? &idx : nullptr, &rho, r,
+                        &Gc, ldgc, nullptr, ws, ws_bytes, PlanOpts(), s);
+  if (dt != GRASS_F32) return GRASS_ERR_UNSUPPORTED;
+  return project_fp32(dY, lddy, X, ldx, T, m, n, idx, rho, r, Gc, ldgc, ws, ws_bytes, s);
+}
 
 extern "C" size_t grass_project_batched_workspace_bytes(int32_t count, int64_t T, int64_t m,
                                                         int64_t n, int32_t r) {
-  (void)m;
-  if (count < 1 || count > grass::kTcMaxGroup || T < 1 || n < 1 || r < 1) return 0;
-  const grass::TcPlan plan = grass::make_plan(T, n, r, false, count);
-  return (plan.ag_bytes + plan.part_bytes) * static_cast<size_t>(count) + 256;
+  if (count < 1 || count > grass::kTcMaxGroup || T < 1 || m < 1 || n < 1 || r < 1) return 0;
+  const grass::TcPlan plan = grass::make_plan(T, m, n, r, true, grass::PlanOpts(), false, count);
+  return grass::plan_ws_bytes(plan, count) + 256;
 }
 
 extern "C" int grass_project_grad_batched(int32_t count, const void* const* dY, int64_t lddy,
@@ -478,21 +570,41 @@ extern "C" int grass_project_grad_batched(int32_t count, const void* const* dY, 
                                           int64_t n, const int32_t* const* idx,
                                           const float* const* rho, int32_t r, float* const* Gc,
                                           int64_t ldgc, void* ws, size_t ws_bytes, void* stream) {
+  return grass_project_grad_ex(count, dY, lddy, X, ldx, T, m, n, idx, rho, r, Gc, ldgc, ws, ws_bytes,
+                               nullptr, stream);
+}
+
+extern "C" int grass_project_plan(int32_t count, int64_t T, int64_t m, int64_t n, int32_t r,
+                                  const grass_project_opts_t* opts, grass_project_plan_t* plan) {
+  using namespace grass;
+  if (plan == nullptr || count < 1 || count > kTcMaxGroup || T < 1 || m < 1 || n < 1 || r < 1 ||
+      r > m || T > 0x7fffffffLL || m > 0x7fffffffLL || n > 0x7fffffffLL || !opts_ok(opts))
+    return GRASS_ERR_INVALID_ARG;
+  describe_plan(make_plan(T, m, n, r, true, to_plan_opts(opts), false, count), count, plan);
+  return GRASS_OK;
+}
+
+extern "C" int grass_project_grad_ex(int32_t count, const void* const* dY, int64_t lddy,
+                                     const void* const* X, int64_t ldx, int64_t T, int64_t m,
+                                     int64_t n, const int32_t* const* idx, const float* const* rho,
+                                     int32_t r, float* const* Gc, int64_t ldgc, void* ws,
+                                     size_t ws_bytes, const grass_project_opts_t* opts,
+                                     void* stream) {
   using namespace grass;
   if (count < 1 || count > kTcMaxGroup || dY == nullptr || X == nullptr || idx == nullptr ||
       Gc == nullptr || T < 1 || m < 1 || n < 1 || r < 1 || r > m || lddy < m || ldx < n ||
-      ldgc < n || T > 0x7fffffffLL || m > 0x7fffffffLL || n > 0x7fffffffLL)
+      ldgc < n || T > 0x7fffffffLL || m > 0x7fffffffLL || n > 0x7fffffffLL || !opts_ok(opts))
     return GRASS_ERR_INVALID_ARG;
   for (int g = 0; g < count; ++g)
     if (idx[g] == nullptr) return GRASS_ERR_INVALID_ARG;
   return project_bf16(count, dY, lddy, X, ldx, T, m, n, idx, rho, r, Gc, ldgc, nullptr, ws, ws_bytes,
-                      static_cast<cudaStream_t>(stream));
+                      to_plan_opts(opts), static_cast<cudaStream_t>(stream));
 }
 
 extern "C" size_t grass_grad_row_norms_workspace_bytes(int64_t T, int64_t m, int64_t n, int dt) {
   if (m < 1 || n < 1 || T < 1) return 0;
   if (dt == GRASS_BF16) {
-    const grass::TcPlan plan = grass::make_norms_plan(T, n, static_cast<int>(m));
+    const grass::TcPlan plan = grass::make_norms_plan(T, m, n);
     return (plan.split_k == 1 ? grass::norm_part_bytes(m, n) : plan.part_bytes) + 256;
   }
   return grass::round_up(static_cast<size_t>(m) * n * sizeof(float), 256) +
@@ -509,7 +621,7 @@ extern "C" int grass_grad_row_norms(const void* dY, int64_t lddy, const void* X,
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dt == GRASS_BF16)
     return project_bf16(1, &dY, lddy, &X, ldx, T, m, n, nullptr, nullptr, static_cast<int>(m),
-                        nullptr, 0, norms, ws, ws_bytes, s);
+                        nullptr, 0, norms, ws, ws_bytes, PlanOpts(), s);
   if (dt != GRASS_F32) return GRASS_ERR_UNSUPPORTED;
   // fp32 path: the (small) gradient is formed in the workspace and reduced by grass_row_norms
   if (ws == nullptr || !aligned_to(ws, 256) ||

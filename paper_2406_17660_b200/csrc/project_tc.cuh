@@ -21,10 +21,20 @@
 // tile boundaries; a "TMEM free" barrier returns the accumulators from the epilogue warps to
 // the MMA issuer between tiles.
 //
-// FUSED = true adds eight gather warps that pick the selected dY columns themselves and write
-// them into the B-operand slabs (generic-proxy stores in the swizzled layout, proxy fence,
-// arrive on "full"); the host uses it for small, densely picked tiles, and the gather pre-pass
-// below otherwise.
+// GATHER selects how the selected dY columns reach the B operand:
+//   kGatherNone  the operand is read by TMA from a matrix that already exists (dY itself for
+//                the dense gradient, or the output of the stand-alone gather_cols_kernel);
+//   kGatherCta   eight extra warps pick dY[t, idx_j] themselves and write the bytes into this
+//                CTA's B-operand slabs (generic-proxy stores in the swizzled layout, proxy
+//                fence, arrive on "full"): for small, densely picked tiles;
+//   kGatherCoop  eight extra warps in EVERY CTA of the grid share the gather of the whole launch:
+//                they take (token chunk, column group) items from one queue in the order the
+//                GEMM consumes them, write the picked columns to the token-major operand matrix
+//                in the workspace (it stays in L2) and publish a per-chunk counter; a CTA's TMA
+//                producer waits for the counter of a chunk before it loads from it.  The gather
+//                is done once per launch instead of once per n-tile, and it overlaps the MMAs
+//                instead of preceding them.  Gather warps never wait on anything, so progress
+//                does not depend on which CTAs are resident.
 //
 // Warp roles (320 threads): warp 0 = TMA producer (one lane per slab), warp 1 =
 // TMEM owner + single-thread MMA issuer, warps 2..9 = epilogue (warp w reads
@@ -80,6 +90,15 @@ __host__ __device__ constexpr int tc_stages(int MB, int A_SLABS) {
 
 constexpr int kTcMaxGroup = 8;
 
+constexpr int kGatherNone = 0, kGatherCta = 1, kGatherCoop = 2;
+// Cooperative gather: tokens per chunk (one readiness counter each), columns per item, and the
+// parts (one warp each) a chunk's tokens are dealt into.  Token slices of the GEMM start on
+// chunk borders in this mode.
+constexpr int kCoopChunk = 128;
+constexpr int kCoopCols = 256;
+constexpr int kCoopParts = 16;
+constexpr int kCoopCtrlInts = 64;     // control block: [0] queue head, flags from [kCoopCtrlInts]
+
 // The X and gathered-dY tensor maps of every layer of the group (kernel parameter space).
 struct TcMaps {
   CUtensorMap x[kTcMaxGroup];
@@ -90,6 +109,7 @@ struct TcParams {
   int T, n, r;          // logical sizes
   int k_blocks;         // ceil(T / tokens per stage)
   int split_k;          // token slices per layer
+  int kb_unit;          // slices start on multiples of this many token blocks
   int tiles_x, tiles_y, tiles_z;   // tile space: n-tiles (per pair if PAIR), row blocks,
                                    // layers * split_k
   // Up to kTcMaxGroup same-shaped layers share one launch: blockIdx.z = group * split_k + split.
@@ -102,6 +122,13 @@ struct TcParams {
   const int32_t* idx[kTcMaxGroup];
   long long lddy;
   int m;
+  // cooperative gather: operand matrices [T][r_pad] being filled, control block, item space
+  __nv_bfloat16* Ag[kTcMaxGroup];
+  int r_pad;
+  int* coop_ctrl;
+  int coop_chunks;      // chunks per layer = ceil(T / kCoopChunk)
+  int coop_cg;          // column groups = ceil(r_pad / kCoopCols)
+  int coop_pmax;        // most chunks in one token slice
   float* norm_part;     // non-NULL: row-norm mode.  Nothing of D is stored; instead
                         // norm_part[g * ld_norm + j] = sum of D[j, c]^2 over the 32 columns c of group g
   long long ld_norm;
@@ -124,9 +151,47 @@ __device__ __forceinline__ float warp_transpose_sum(float (&x)[32], int lane) {
   return x[0];
 }
 
-template <int MB, int NSLAB, bool PAIR, bool FUSED>
-__global__ void __launch_bounds__(FUSED ? kTcThreads + kTcGatherThreads : kTcThreads, 1)
+// dY[t, rows[i]] for 32 (token, column) pairs per lane in flight, written to the operand matrix.
+// Lane l carries columns col0 + 32 i + l, i < NI; tokens tok0, tok0 + kCoopParts, ...
+template <int NI>
+__device__ __forceinline__ void coop_gather_part(const unsigned short* __restrict__ src,
+                                                 long long lddy, unsigned short* __restrict__ dst,
+                                                 int r_pad, int col0, const int (&rows)[8], int tok0,
+                                                 int T, int lane) {
+  constexpr int TU = (32 / NI) < (kCoopChunk / kCoopParts) ? (32 / NI) : (kCoopChunk / kCoopParts);   // tokens per batch of loads
+  constexpr int NTOK = kCoopChunk / kCoopParts;           // tokens of this part
+  // Every load is unconditional (rows and tokens clamped to valid ones, the value discarded at
+  // the store): a load under a per-lane condition would be followed by a select on its result,
+  // and the warp would wait for each load before issuing the next.
+  int safe[NI];
+#pragma unroll
+  for (int i = 0; i < NI; ++i) safe[i] = rows[i] >= 0 ? rows[i] : 0;
+#pragma unroll 1
+  for (int k0 = 0; k0 < NTOK; k0 += TU) {
+    unsigned short v[TU][NI];
+#pragma unroll
+    for (int u = 0; u < TU; ++u) {
+      const int tok = tok0 + (k0 + u) * kCoopParts;
+      const unsigned short* line = src + static_cast<long long>(tok < T ? tok : T - 1) * lddy;
+#pragma unroll
+      for (int i = 0; i < NI; ++i) v[u][i] = ptx::ld_nc_na_u16(line + safe[i]);
+    }
+#pragma unroll
+    for (int u = 0; u < TU; ++u) {
+      const int tok = tok0 + (k0 + u) * kCoopParts;
+      unsigned short* out = dst + static_cast<long long>(tok) * r_pad + col0 + lane;
+#pragma unroll
+      for (int i = 0; i < NI; ++i)
+        if (tok < T && col0 + 32 * i + lane < r_pad) out[32 * i] = rows[i] >= 0 ? v[u][i] : 0;
+    }
+  }
+}
+
+template <int MB, int NSLAB, bool PAIR, int GATHER>
+__global__ void __launch_bounds__(GATHER != kGatherNone ? kTcThreads + kTcGatherThreads : kTcThreads, 1)
 project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
+  constexpr bool FUSED = GATHER == kGatherCta;
+  constexpr bool COOP = GATHER == kGatherCoop;
   constexpr int R_CTA = 64 * NSLAB;          // selected rows per CTA tile (per pair if PAIR)
   constexpr int X_SLABS = 2 * MB;
   constexpr int A_SLABS = PAIR ? NSLAB / 2 : NSLAB;   // slabs of the gathered operand this CTA stages
@@ -166,7 +231,9 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   const int n_workers = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
   const int worker = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
   const int n_tiles = p.tiles_x * p.tiles_y * p.tiles_z;
-  const int kb_per = p.k_blocks / p.split_k, kb_rem = p.k_blocks % p.split_k;
+  // token slices in units of kb_unit blocks: u_per or u_per + 1 units each
+  const int n_units = (p.k_blocks + p.kb_unit - 1) / p.kb_unit;
+  const int u_per = n_units / p.split_k, u_rem = n_units % p.split_k;
 
   // decode a linear tile index (identical in every role)
   struct Tile { int c_base, r0, grp, z, kb_begin, kb_count; };
@@ -181,8 +248,9 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     t.r0 = by * R_CTA;
     t.grp = bz / p.split_k;                 // which layer of the group
     t.z = bz - t.grp * p.split_k;           // which token slice
-    t.kb_begin = t.z * kb_per + (t.z < kb_rem ? t.z : kb_rem);
-    t.kb_count = kb_per + (t.z < kb_rem ? 1 : 0);
+    t.kb_begin = (t.z * u_per + (t.z < u_rem ? t.z : u_rem)) * p.kb_unit;
+    t.kb_count = (u_per + (t.z < u_rem ? 1 : 0)) * p.kb_unit;
+    if (t.kb_begin + t.kb_count > p.k_blocks) t.kb_count = p.k_blocks - t.kb_begin;
     return t;
   };
 
@@ -236,8 +304,46 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         xcoord = t.r0 + (lane - X_SLABS) * 64;
       }
       int tok = t.kb_begin * kTcBK;
+      int ready_upto = 0;        // COOP: chunks below this one are known to be complete
+      const int chunk_end = (t.kb_begin + t.kb_count) * kTcBK / kCoopChunk +
+                            (((t.kb_begin + t.kb_count) * kTcBK) % kCoopChunk != 0 ? 1 : 0);
       for (int it = 0; it < t.kb_count; ++it) {
         int ok = 1;
+        if (COOP && tok / kCoopChunk >= ready_upto) {
+          // The gather warps of the grid publish kCoopParts * coop_cg arrivals per chunk.  One
+          // probe reads the counters of the next 32 chunks of this slice (lane l: chunk + l) and
+          // advances ready_upto over the leading run of complete ones, so that a gather running
+          // ahead costs the producer one L2 round trip per 32 chunks, not one per chunk.
+          const int chunk = tok / kCoopChunk;
+          const int* flags = p.coop_ctrl + kCoopCtrlInts + t.grp * p.coop_chunks;
+          const int want = kCoopParts * p.coop_cg;
+          const long long start = clock64();
+          int n_ready = 0;
+          while (true) {
+            const int c = chunk + lane;
+            const bool done = c < chunk_end && ptx::flag_load_acquire(flags + c) >= want;
+            const uint32_t mask = __ballot_sync(0xffffffffu, done);
+            n_ready = __ffs(~mask) - 1;            // leading run of complete chunks (mask != all ones
+            if (mask == 0xffffffffu) n_ready = 32; // unless every lane saw a complete chunk)
+            if (n_ready > 0) break;
+            __nanosleep(32);
+            int give_up = 0;
+            if (lane == 0) give_up = (*abort_flag != 0 || clock64() - start > kTcWaitLimit) ? 1 : 0;
+            if (__shfl_sync(0xffffffffu, give_up, 0)) break;
+          }
+          if (n_ready == 0) {
+            if (lane == 0) {
+              if (*abort_flag == 0) record_status(p.status, GRASS_ERR_TIMEOUT, 500);
+              *abort_flag = 1;
+            }
+            alive = false;
+            break;
+          }
+          ready_upto = chunk + n_ready;
+          __syncwarp();
+          // generic-proxy stores of other SMs (acquired above) -> this warp's TMA reads
+          ptx::fence_proxy_async_global();
+        }
         if (lane == 0) {
           ok = ptx::mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kTcWaitLimit) ? 1 : 0;
           if (ok) {
@@ -330,6 +436,69 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         if (!ok) ptx::mbar_wait_bounded(&bar_accum, tile_ph, nullptr, kTcDrainLimit);
         tile_ph ^= 1u;
       }
+    }
+  } else if (COOP && warp >= kTcThreads / 32) {
+    // ================= gather warps (COOP): shared queue over the whole launch =================
+    // Item = (token slice bz, chunk position pp in the slice, column group, part): one warp
+    // copies dY[t, idx[j]] for the part's 16 tokens and up to 256 columns j into Ag[t, j].
+    // Queue order follows the GEMM: slices grouped by the wave of tiles that first touches them,
+    // inside a group chunk position first, so every running tile finds its next chunk early.
+    // Padding items (a slice shorter than coop_pmax) are skipped.
+    const int txy = p.tiles_x * p.tiles_y;
+    const int n_waves = (n_tiles + n_workers - 1) / n_workers;
+    const int per_chunk = p.coop_cg * kCoopParts;
+    const int per_slice = p.coop_pmax * per_chunk;
+    const int total = p.tiles_z * per_slice;
+    while (true) {
+      int q = 0;
+      if (lane == 0) q = atomicAdd(p.coop_ctrl, 1);
+      q = __shfl_sync(0xffffffffu, q, 0);
+      if (q >= total) break;
+      int bz_lo = 0, bz_hi = 0, base = 0;
+      for (int w = 0; w < n_waves; ++w) {
+        const int last_tile = ((w + 1) * n_workers < n_tiles ? (w + 1) * n_workers : n_tiles) - 1;
+        bz_hi = last_tile / txy + 1;
+        const int items = (bz_hi - bz_lo) * per_slice;
+        if (q < base + items || w == n_waves - 1) break;
+        base += items;
+        bz_lo = bz_hi;
+      }
+      const int in_wave = q - base, cnt = bz_hi - bz_lo;
+      const int pp = in_wave / (cnt * per_chunk);
+      const int rem = in_wave - pp * (cnt * per_chunk);
+      const int bz = bz_lo + rem / per_chunk;
+      const int rem2 = rem - (rem / per_chunk) * per_chunk;
+      const int cg = rem2 / kCoopParts, part = rem2 - cg * kCoopParts;
+      const int grp = bz / p.split_k, z = bz - grp * p.split_k;
+      const int units = u_per + (z < u_rem ? 1 : 0);
+      if (pp >= units || bz >= p.tiles_z) continue;          // padding item
+      const int chunk = z * u_per + (z < u_rem ? z : u_rem) + pp;   // kb_unit blocks = one chunk
+      const int col0 = cg * kCoopCols;
+      const int32_t* idx = p.idx[grp];
+      int rows[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int j = col0 + 32 * i + lane;
+        int row = -1;
+        if (j < p.r) {
+          row = __ldg(idx + j);
+          if (row < 0 || row >= p.m) {
+            record_status(p.status, GRASS_ERR_INVALID_ARG, row);
+            row = -1;
+          }
+        }
+        rows[i] = row;
+      }
+      const unsigned short* src = reinterpret_cast<const unsigned short*>(p.dY[grp]);
+      unsigned short* dst = reinterpret_cast<unsigned short*>(p.Ag[grp]);
+      const int tok0 = chunk * kCoopChunk + part;
+      const int cols = p.r_pad - col0;
+      if (cols <= 64) coop_gather_part<2>(src, p.lddy, dst, p.r_pad, col0, rows, tok0, p.T, lane);
+      else if (cols <= 128) coop_gather_part<4>(src, p.lddy, dst, p.r_pad, col0, rows, tok0, p.T, lane);
+      else coop_gather_part<8>(src, p.lddy, dst, p.r_pad, col0, rows, tok0, p.T, lane);
+      __threadfence();           // this lane's stores are performed device-wide ...
+      __syncwarp();
+      if (lane == 0) ptx::flag_arrive_release(p.coop_ctrl + kCoopCtrlInts + grp * p.coop_chunks + chunk);
     }
   } else if (FUSED && warp >= kTcThreads / 32) {
     // ================= gather warps (FUSED): dY[t, idx[j]] -> swizzled B-operand slabs =================

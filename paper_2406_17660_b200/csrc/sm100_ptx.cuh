@@ -80,6 +80,28 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
   }
 }
 
+// ---- cross-CTA hand-over through global memory (cooperative gather) ----
+// Producer side: after its data stores and a __threadfence, one lane adds 1 to the counter.
+__device__ __forceinline__ void flag_arrive_release(int* flag) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(flag) : "memory");
+}
+__device__ __forceinline__ int flag_load_acquire(const int* flag) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+  return v;
+}
+// Data written with ordinary stores by other SMs, then acquired through a flag, is about to be
+// read by this thread's TMA copies (async proxy).
+__device__ __forceinline__ void fence_proxy_async_global() {
+  asm volatile("fence.proxy.async.global;" ::: "memory");
+}
+// 16-bit read-only load that does not allocate in L1 (each selected column is read once).
+__device__ __forceinline__ unsigned short ld_nc_na_u16(const unsigned short* p) {
+  unsigned short v;
+  asm volatile("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(v) : "l"(p));
+  return v;
+}
+
 // ---- TMA: 2-D tiled load, global -> shared, completion on an mbarrier ----
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y,
                                             uint64_t* bar) {

@@ -212,7 +212,7 @@ def test_select_degenerate_inputs_leave_outputs_untouched():
 
 # --------------------------------------------------------------------------- projection
 def _project_case(T, m, n, r, dtype, seed, ldx=None, lddy=None, identity=False, dup=False,
-                  with_rho=True):
+                  with_rho=True, opts=None):
     X = syn.make_X(T, n, dtype, seed0=seed, ld=ldx)
     dY = syn.make_dY(T, m, dtype, seed0=seed, ld=lddy)
     rng = np.random.default_rng(seed)
@@ -228,11 +228,28 @@ def _project_case(T, m, n, r, dtype, seed, ldx=None, lddy=None, identity=False, 
     dYd = syn._padded(dY.to(DEV), lddy or m)
     Gc = torch.full((r, n), float("nan"), dtype=torch.float32, device=DEV)
     dt = grass.BF16 if dtype == torch.bfloat16 else grass.F32
-    ws = ws_bytes(grass.grass_project_workspace_bytes(T, m, n, r, dt))
-    grass.grass_project_grad(dYd, Xd, idx_t, rho_t, r, Gc, ws)
+    if opts is None:
+        ws = ws_bytes(grass.grass_project_workspace_bytes(T, m, n, r, dt))
+        grass.grass_project_grad(dYd, Xd, idx_t, rho_t, r, Gc, ws)
+    else:
+        plan = grass.grass_project_plan(1, T, m, n, r, opts)
+        ws = ws_bytes(plan["workspace_bytes"])
+        ws.fill_(0xA5)                       # the library must not rely on a clean workspace
+        grass.grass_project_grad_ex([dYd], [Xd], [idx_t], None if rho_t is None else [rho_t], r,
+                                    [Gc], ws, opts)
     grass.grass_device_status()
     want = oracle.project_grad(f64(dY), f64(X), sigma, rho_np)
     return f64(Gc), want
+
+
+def _assert_close_gc(got, want, tol=1e-4):
+    """Frobenius bound (the acceptance metric) plus an element-wise bound that localises a bad
+    tile: no element off by more than tol of the largest expected magnitude."""
+    assert np.all(np.isfinite(got))
+    err = rel_fro(got, want)
+    assert err <= tol, err
+    worst = np.max(np.abs(got - want))
+    assert worst <= tol * np.max(np.abs(want)), worst
 
 
 @pytest.mark.parametrize("T,m,n,r", [(512, 256, 256, 32), (100, 50, 70, 7), (33, 65, 129, 65)])
@@ -581,25 +598,52 @@ def test_resume_from_copied_state_is_bit_identical():
 
 
 # --------------------------------------------------------------------------- kernel variants
-@pytest.mark.parametrize("force_mb", ["1", "2", "4"])
-@pytest.mark.parametrize("no_pair", [False, True])
-@pytest.mark.parametrize("no_fused", [False, True])
-def test_every_tile_variant_of_the_projection_kernel(force_mb, no_pair, no_fused, monkeypatch):
+@pytest.mark.parametrize("mb", [1, 2, 4])
+@pytest.mark.parametrize("pair", [grass.PAIR_NEVER, grass.PAIR_ALWAYS])
+@pytest.mark.parametrize("gather", [grass.GATHER_PREPASS, grass.GATHER_IN_CTA, grass.GATHER_COOPERATIVE])
+def test_every_tile_variant_of_the_projection_kernel(mb, pair, gather):
     """The host picks the tile shape from a cost model, so a given problem exercises one template
-    instantiation.  The diagnostic switches pin the n-blocks per CTA, single CTAs instead of CTA
-    pairs, and the gather pre-pass instead of the in-kernel gather, so that every instantiation
-    that can serve these shapes is run and checked against the oracle."""
-    monkeypatch.setenv("GRASS_TC_FORCE_MB", force_mb)
-    if no_pair:
-        monkeypatch.setenv("GRASS_TC_NO_PAIR", "1")
-    if no_fused:
-        monkeypatch.setenv("GRASS_TC_NO_FUSED_GATHER", "1")
-    monkeypatch.setenv("GRASS_TC_FUSED_MAX_TILES", "8")
+    instantiation.  Explicit options pin the n-blocks per CTA, single CTAs or CTA pairs, and the
+    way the selected columns reach the GEMM (pre-pass, in-CTA gather, cooperative gather), so
+    that every instantiation that can serve these shapes is run and checked against the oracle."""
+    opts = dict(gather=gather, n_blocks_per_cta=mb, cta_pair=pair)
+    seen = set()
     for T, m, n, r in [(1500, 512, 1024, 128), (900, 256, 520, 64), (1100, 640, 1024, 256),
                        (800, 1200, 1024, 448)]:
-        got, want = _project_case(T, m, n, r, torch.bfloat16, seed=T + r, dup=True)
-        err = rel_fro(got, want)
-        assert np.all(np.isfinite(got)) and err <= 1e-4, (T, m, n, r, err)
+        plan = grass.grass_project_plan(1, T, m, n, r, opts)
+        seen.add((plan["gather"], plan["n_blocks_per_cta"], plan["cta_pair"], plan["rows_per_tile"]))
+        got, want = _project_case(T, m, n, r, torch.bfloat16, seed=T + r, dup=True, opts=opts)
+        _assert_close_gc(got, want)
+    assert len(seen) >= 3
+
+
+@pytest.mark.parametrize("slices", [1, 2, 3, 7])
+@pytest.mark.parametrize("T,m,n,r", [(2000, 512, 768, 192), (4100, 2048, 1024, 1024), (129, 300, 256, 40)])
+def test_cooperative_gather_over_token_slices(T, m, n, r, slices):
+    """Cooperative gather with the token sum cut into 1..7 slices (slices start on 128-token
+    chunk borders; ragged last chunk; r not a multiple of the column group)."""
+    opts = dict(gather=grass.GATHER_COOPERATIVE, token_slices=slices)
+    got, want = _project_case(T, m, n, r, torch.bfloat16, seed=T + r + slices, opts=opts)
+    _assert_close_gc(got, want)
+
+
+def test_cooperative_gather_is_bit_reproducible_and_matches_the_prepass():
+    """Same tiling, same token slices: the cooperative gather and the pre-pass feed the GEMM the
+    same operand bits, so the results are identical, run after run."""
+    T, m, n, r = 3072, 2048, 1024, 512        # 24 chunks of 128 tokens: both cut it 16/16/16 blocks
+    X = syn.make_X(T, n, torch.bfloat16, seed0=9).to(DEV)
+    dY = syn.make_dY(T, m, torch.bfloat16, seed0=9).to(DEV)
+    idx = torch.tensor(np.sort(np.random.default_rng(1).choice(m, r, replace=False)),
+                       dtype=torch.int32, device=DEV)
+    outs = []
+    for gather in (grass.GATHER_COOPERATIVE, grass.GATHER_COOPERATIVE, grass.GATHER_PREPASS):
+        opts = dict(gather=gather, token_slices=3)
+        ws = ws_bytes(grass.grass_project_plan(1, T, m, n, r, opts)["workspace_bytes"])
+        Gc = torch.empty((r, n), dtype=torch.float32, device=DEV)
+        grass.grass_project_grad_ex([dY], [X], [idx], None, r, [Gc], ws, opts)
+        grass.grass_device_status()
+        outs.append(Gc)
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
 
 
 def test_updates_with_repeated_rows_are_bit_reproducible():
