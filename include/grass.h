@@ -279,6 +279,8 @@ int grass_adam_scatter_batched(int32_t count, const float* const* Gc, int64_t ld
  *                     accumulators would not fit).
  *   cta_pair          GRASS_PAIR_NEVER / GRASS_PAIR_ALWAYS (where r allows it).
  *   token_slices      number of slices of T (clamped to what T allows).
+ *   gather_warps      GRASS_GATHER_COOPERATIVE only: how many of a CTA's eight gather
+ *                     warps take part (1..8).
  * grass_project_plan reports what a call with these arguments would do, and the
  * workspace it needs, without touching the GPU (plan: host pointer, written).
  * grass_project_grad_ex takes the arguments of grass_project_grad_batched plus
@@ -292,6 +294,7 @@ typedef struct {
   int32_t n_blocks_per_cta;
   int32_t cta_pair;
   int32_t token_slices;
+  int32_t gather_warps;
 } grass_project_opts_t;
 typedef struct {
   int32_t gather;            /* GRASS_GATHER_* actually used */
@@ -300,7 +303,9 @@ typedef struct {
   int32_t n_blocks_per_cta;
   int32_t ctas_per_slice;    /* CTAs that share one token slice, over all `count` layers */
   int32_t cta_pair;          /* 1: two CTAs per MMA */
-  int32_t token_slices;
+  int32_t token_slices;      /* slices of T, each summed into its own fp32 partial */
+  int32_t short_slices;      /* how many of them are the short slices that fill the last wave */
+  int32_t long_slice_tokens; /* tokens in the first slice */
   int32_t tokens_per_stage;  /* tokens per pipeline stage (32 or 64) */
   int32_t stages;
   size_t workspace_bytes;

@@ -313,14 +313,15 @@ PAIR_AUTO, PAIR_NEVER, PAIR_ALWAYS = 0, 1, 2
 class ProjectOpts(ctypes.Structure):
     """grass_project_opts_t: 0 in a field keeps the library's own choice."""
     _fields_ = [("gather", c_int32), ("n_blocks_per_cta", c_int32), ("cta_pair", c_int32),
-                ("token_slices", c_int32)]
+                ("token_slices", c_int32), ("gather_warps", c_int32)]
 
 
 class ProjectPlan(ctypes.Structure):
     """grass_project_plan_t."""
     _fields_ = [("gather", c_int32), ("rows_per_tile", c_int32), ("row_blocks", c_int32),
                 ("n_blocks_per_cta", c_int32), ("ctas_per_slice", c_int32), ("cta_pair", c_int32),
-                ("token_slices", c_int32), ("tokens_per_stage", c_int32), ("stages", c_int32),
+                ("token_slices", c_int32), ("short_slices", c_int32), ("long_slice_tokens", c_int32),
+                ("tokens_per_stage", c_int32), ("stages", c_int32),
                 ("workspace_bytes", c_size_t)]
 
 

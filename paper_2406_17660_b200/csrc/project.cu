@@ -21,6 +21,7 @@ struct PlanOpts {
   int mb = 0;              // n-blocks of 128 columns per CTA: 0 = cost model, else 1, 2 or 4 if it fits
   int pair = 0;            // 0 = cost model, 1 = single CTAs only, 2 = CTA pairs wherever the shape allows
   int split = 0;           // token slices: 0 = cost model
+  int gather_warps = 0;    // cooperative gather: warps per CTA that gather (0 = default)
 };
 
 PlanOpts to_plan_opts(const grass_project_opts_t* o) {
@@ -30,6 +31,7 @@ PlanOpts to_plan_opts(const grass_project_opts_t* o) {
     po.mb = o->n_blocks_per_cta;
     po.pair = o->cta_pair;
     po.split = o->token_slices;
+    po.gather_warps = o->gather_warps;
   }
   return po;
 }
@@ -38,7 +40,8 @@ bool opts_ok(const grass_project_opts_t* o) {
          (o->gather >= kOptAuto && o->gather <= kOptCoop &&
           (o->n_blocks_per_cta == 0 || o->n_blocks_per_cta == 1 || o->n_blocks_per_cta == 2 ||
            o->n_blocks_per_cta == 4) &&
-          o->cta_pair >= 0 && o->cta_pair <= 2 && o->token_slices >= 0);
+          o->cta_pair >= 0 && o->cta_pair <= 2 && o->token_slices >= 0 &&
+          o->gather_warps >= 0 && o->gather_warps <= 8);
 }
 
 struct TcPlan {
@@ -47,20 +50,50 @@ struct TcPlan {
   size_t ctrl_bytes;   // cooperative gather: queue head and per-chunk counters
   int r_pad;      // r_blocks * r_cta: width of the gathered operand
   int r_cta, r_blocks;
-  int MB, n_blocks;   // n_blocks = gridDim.x (CTAs, an even number when pair)
+  int MB, n_blocks;   // n_blocks = CTAs along n (an even number when pair)
   bool pair;          // two CTAs share each MMA (cta_group::2)
-  int k_blocks, split_k, stages, bk;   // bk: tokens per pipeline stage
+  int k_blocks, stages, bk;   // bk: tokens per pipeline stage
+  int split_k, s_long;        // token slices; the first s_long are long, the rest short
+  int unit_begin[kTcMaxSlices + 1];   // slice z = units [unit_begin[z], unit_begin[z + 1])
   size_t smem_bytes;
   long long ld_part;        // pitch of a split-K partial, elements
   size_t ag_bytes, part_bytes;
 };
 
-// Choose the CTA tile and the token split.  Cost model in SM clocks: the MMA
-// phase takes waves * (token blocks per CTA * clocks per block + prologue and
-// epilogue), and split-K partials cost their HBM write plus re-read.  Smaller
-// n-tiles (MB) make more, smaller CTAs, which cuts partial traffic when the
-// output is tiny; larger ones cut the number of times the gathered operand is
-// re-read.  The result depends only on (T, n, r), so it is reproducible.
+// How the selected columns get to the GEMM for a given tile shape.  In-CTA gather: the GEMM's
+// own warps pick the columns out of dY into shared memory.  It pays when a tile holds at most
+// 128 rows (the load unit keeps up), at most two CTAs (pairs) share a token slice (each gathers
+// for itself) and the picks are dense enough that a 32-lane load spans at most 6 cache lines
+// (12 r >= m); measured on the 60M q,k,v,o group (m = 512, r = 128): step 253 -> 274 TFLOP/s,
+// while at m = 2048, r = 128 the sparser pick made the in-kernel loads the bottleneck.
+// Everything else: cooperative gather (all CTAs share one pass over dY, overlapped with the
+// MMAs); the stand-alone pre-pass remains selectable.
+int choose_gather(bool has_idx, const PlanOpts& opts, int r_cta, int tiles_x, int64_t m, int r) {
+  if (!has_idx) return 0;
+  const bool cta_ok = r_cta <= 128;
+  if (opts.gather == kOptCta && cta_ok) return kOptCta;
+  if (opts.gather == kOptPrepass) return kOptPrepass;
+  if (opts.gather == kOptCoop) return kOptCoop;
+  if (opts.gather == kOptAuto && cta_ok && tiles_x <= 2 && static_cast<int64_t>(r) * 12 >= m)
+    return kOptCta;
+  return kOptCoop;
+}
+
+// Choose the CTA tile and the token slices.  Cost model in SM clocks.  A worker (a CTA, or a
+// CTA pair) needs `c` clocks per unit of tokens and `f` clocks per tile (pipeline fill,
+// epilogue).  With N = tiles-per-slice x slices tiles on W workers the time is that of the
+// busiest worker; equal slices leave the last wave partly empty whenever W does not divide N.
+// So besides s_long equal slices the search tries up to three extra SHORT slices: the
+// R = N_long mod W workers that receive one long tile more than the rest are then finished,
+// and the other W - R workers share the short tiles; the lengths (x units long, y units short)
+// are set so that both kinds of worker finish together:
+//     x c + f = ns (y c + f),  s_long x + s_short y = U,  ns = ceil(N_short / (W - R)).
+// The operands reach the SMs from L2 (every CTA fetches its own tiles): the X tile of an n-block
+// once per row block and the gathered operand once per n-tile.  On the LLaMA-7B r = 1024 shapes
+// this traffic (about 8.6 TB/s), not the number of busy SMs, bounds the kernel: the same 187 us
+// with 128 or with all 148 SMs at work.  Split-K partials cost their HBM write plus re-read.  Smaller n-tiles (MB) make more,
+// smaller CTAs, which cuts partial traffic when the output is tiny; larger ones cut the number
+// of times the gathered operand is re-read.  The result depends only on the arguments.
 TcPlan make_plan(int64_t T, int64_t m, int64_t n, int r, bool has_idx, const PlanOpts& opts,
                  bool single_split = false, int groups = 1) {
   TcPlan p;
@@ -68,7 +101,6 @@ TcPlan make_plan(int64_t T, int64_t m, int64_t n, int r, bool has_idx, const Pla
   p.r_blocks = (r64 + 511) / 512;
   p.r_cta = static_cast<int>(round_up(static_cast<size_t>((r64 + p.r_blocks - 1) / p.r_blocks), 64));
   p.r_pad = p.r_cta * p.r_blocks;
-  p.k_blocks = static_cast<int>((T + 31) / 32);   // in 32-token units while searching
   int mb_max = 512 / p.r_cta;
   mb_max = mb_max >= 4 ? 4 : (mb_max >= 2 ? 2 : 1);
   while (mb_max > 1 && static_cast<int64_t>(mb_max / 2) * 128 >= n) mb_max /= 2;  // not past n
@@ -76,71 +108,107 @@ TcPlan make_plan(int64_t T, int64_t m, int64_t n, int r, bool has_idx, const Pla
   const double hbm_bytes_per_clk = 6.5e12 / 1.7e9;  // whole chip, per SM clock
   double best = 1e300;
   p.MB = 1;
-  p.split_k = 1;
-  const int force_mb = opts.mb;
-  const bool can_pair = (p.r_cta % 128) == 0 && opts.pair != 1;
   p.pair = false;
+  p.split_k = p.s_long = 1;
+  int best_x = 0;            // units per long slice (0: equal slices)
+  const bool can_pair = (p.r_cta % 128) == 0 && opts.pair != 1;
   for (int mb = mb_max; mb >= 1; mb /= 2) {
-    if (force_mb > 0 && force_mb <= mb_max && mb != force_mb) continue;
+    if (opts.mb > 0 && opts.mb <= mb_max && mb != opts.mb) continue;
     for (int pair = can_pair ? 1 : 0; pair >= 0; --pair) {
       if (pair && n <= static_cast<int64_t>(mb) * 128) continue;  // nothing for the second CTA
       if (!pair && opts.pair == 2 && can_pair && n > static_cast<int64_t>(mb) * 128) continue;
       const int cta_cols = mb * 128 * (pair ? 2 : 1);
-      const int n_tiles = static_cast<int>((n + cta_cols - 1) / cta_cols);
-      const int64_t tiles =
-          static_cast<int64_t>(n_tiles) * p.r_blocks * (pair ? 2 : 1) * groups;  // CTAs per split
-      // clocks per 32-token block: tensor time, or (single CTA) the shared-memory ceiling
-      double clk_per_block = static_cast<double>(mb) * p.r_cta;
-      if (!pair) clk_per_block *= 1.4;
-      if (clk_per_block < 256.0) clk_per_block = 256.0;
-      const double fixed = 3000.0 + mb * 128.0 * p.r_cta * 4.0 / 128.0;
-      const int max_s = single_split ? 1 : (p.k_blocks < 256 ? p.k_blocks : 256);
-      for (int s = 1; s <= max_s; ++s) {
-        if (opts.split > 0 && !single_split && s != (opts.split < max_s ? opts.split : max_s)) continue;
-        const int64_t ctas = tiles * s;
-        const int64_t waves = (ctas + kSmCount - 1) / kSmCount;
-        const double blocks_per_cta = static_cast<double>((p.k_blocks + s - 1) / s);
-        double cost = waves * (blocks_per_cta * clk_per_block + fixed);
-        if (s > 1) cost += 8.0 * s * groups * static_cast<double>(r) * n / hbm_bytes_per_clk;
-        if (cost < best) {
-          best = cost;
-          p.MB = mb;
-          p.split_k = s;
-          p.pair = pair != 0;
+      const int tiles_x = static_cast<int>((n + cta_cols - 1) / cta_cols);
+      const int64_t n_out = static_cast<int64_t>(tiles_x) * p.r_blocks * groups;   // tiles per slice
+      const int W = pair ? kSmCount / 2 : kSmCount;
+      const int a_slabs = pair ? p.r_cta / 128 : p.r_cta / 64;
+      const int bk = tc_bk(mb, a_slabs);
+      const int gather = choose_gather(has_idx, opts, p.r_cta, tiles_x, m, r);
+      const int unit_tokens = gather == kOptCoop ? kCoopChunk : bk;
+      const int U = static_cast<int>((T + unit_tokens - 1) / unit_tokens);
+      // clocks per 32 tokens of one CTA: tensor time, or (single CTA) the shared-memory ceiling;
+      // never less than 256 (a CTA cannot stream its operands faster)
+      double c = static_cast<double>(mb) * p.r_cta;
+      if (!pair) c *= 1.4;
+      if (c < 256.0) c = 256.0;
+      c *= unit_tokens / 32.0;
+      const double f = 3000.0 + mb * 128.0 * p.r_cta * 4.0 / 128.0;   // pipeline fill, accumulator drain
+      // L2 -> SM bytes of the whole launch (per CTA and 32 tokens: (columns + rows) x 64 bytes) at
+      // about 8.6 TB/s.  It overlaps the MMAs only in part: half of it is charged, which is what
+      // makes wider n-tiles (fewer re-reads of the gathered operand) win on the HBM-bound shapes.
+      const double cta_rows = pair ? p.r_cta / 2 : p.r_cta;
+      const double l2_clk = static_cast<double>(tiles_x) * p.r_blocks * groups * (pair ? 2 : 1) *
+                            static_cast<double>((T + 31) / 32) * (mb * 128.0 + cta_rows) * 64.0 / 4500.0;
+      const int max_s = single_split ? 1 : (U < kTcMaxSlices ? U : kTcMaxSlices);
+      for (int sl = 1; sl <= max_s; ++sl) {
+        if (opts.split > 0 && !single_split && sl != (opts.split < max_s ? opts.split : max_s)) continue;
+        const int64_t n_long = n_out * sl;
+        const int64_t F = n_long / W, R = n_long % W;
+        // short slices where they were measured to pay: launches of three or more waves
+        // (7B down, r = 1024: 587 -> 539 us), and the in-CTA gather, where each worker is bound
+        // by its own gather warps (60M q,k,v,o: 179 -> 155 us).  With fewer waves the kernel is
+        // bound by operand traffic, and the extra partials cost more than the idle SMs.
+        const int max_short =
+            (single_split || opts.split > 0 || R == 0 || (F < 2 && gather != kOptCta)) ? 0 : 3;
+        for (int ss = 0; ss <= max_short && sl + ss <= max_s; ++ss) {
+          double span;
+          int x_units = 0;
+          if (ss == 0) {
+            span = static_cast<double>((n_long + W - 1) / W) * (((U + sl - 1) / sl) * c + f);
+          } else {
+            const int64_t ns = (n_out * ss + (W - R) - 1) / (W - R);
+            const double x = (U + ss * (f / c) * (1.0 - 1.0 / ns)) / (sl + static_cast<double>(ss) / ns);
+            span = 1e300;
+            for (int cand = static_cast<int>(x); cand <= static_cast<int>(x) + 1; ++cand) {
+              const int y_total = U - sl * cand;
+              if (cand < 1 || y_total < ss) continue;
+              const int y_max = (y_total + ss - 1) / ss;
+              const double a = (F + 1) * (cand * c + f);
+              const double b = F * (cand * c + f) + ns * (y_max * c + f);
+              const double sp = a > b ? a : b;
+              if (sp < span) { span = sp; x_units = cand; }
+            }
+            if (x_units == 0) continue;
+          }
+          double cost = span + 0.5 * l2_clk;
+          if (sl + ss > 1) cost += 8.0 * (sl + ss) * groups * static_cast<double>(r) * n / hbm_bytes_per_clk;
+          if (cost < best) {
+            best = cost;
+            p.MB = mb;
+            p.pair = pair != 0;
+            p.s_long = sl;
+            p.split_k = sl + ss;
+            best_x = x_units;
+          }
         }
       }
     }
   }
-  {
-    const int cta_cols = p.MB * 128 * (p.pair ? 2 : 1);
-    p.n_blocks = static_cast<int>((n + cta_cols - 1) / cta_cols) * (p.pair ? 2 : 1);
-  }
+  const int cta_cols = p.MB * 128 * (p.pair ? 2 : 1);
+  const int tiles_x = static_cast<int>((n + cta_cols - 1) / cta_cols);
+  p.n_blocks = tiles_x * (p.pair ? 2 : 1);
   const int a_slabs = p.pair ? p.r_cta / 128 : p.r_cta / 64;
   p.bk = tc_bk(p.MB, a_slabs);
   p.k_blocks = static_cast<int>((T + p.bk - 1) / p.bk);
-  // How the selected columns get to the GEMM.  In-CTA gather: the GEMM's own warps pick the
-  // columns out of dY into shared memory.  It pays when a tile holds at most 128 rows (the load
-  // unit keeps up), at most two CTAs (pairs) share a token slice (each gathers for itself) and
-  // the picks are dense enough that a 32-lane load spans at most 6 cache lines (12 r >= m);
-  // measured on the 60M q,k,v,o group (m = 512, r = 128): step 253 -> 274 TFLOP/s, while at
-  // m = 2048, r = 128 the sparser pick made the in-kernel loads the bottleneck (471 -> 379).
-  // Everything else: cooperative gather (all CTAs share one pass over dY, overlapped with the
-  // MMAs); the stand-alone pre-pass remains selectable.
-  p.gather = 0;
-  if (has_idx) {
-    const int tiles_x = p.pair ? p.n_blocks / 2 : p.n_blocks;
-    const bool cta_ok = p.r_cta <= 128;
-    if (opts.gather == kOptCta && cta_ok) p.gather = kOptCta;
-    else if (opts.gather == kOptPrepass) p.gather = kOptPrepass;
-    else if (opts.gather == kOptCoop) p.gather = kOptCoop;
-    else if (opts.gather == kOptAuto && cta_ok && tiles_x <= 2 && static_cast<int64_t>(r) * 12 >= m)
-      p.gather = kOptCta;
-    else p.gather = kOptCoop;
-  }
+  p.gather = choose_gather(has_idx, opts, p.r_cta, tiles_x, m, r);
   p.kb_unit = p.gather == kOptCoop ? kCoopChunk / p.bk : 1;
   {
-    const int n_units = (p.k_blocks + p.kb_unit - 1) / p.kb_unit;
-    if (p.split_k > n_units) p.split_k = n_units;
+    // slice table: long slices of best_x units (or an equal cut), then the short ones
+    const int U = (p.k_blocks + p.kb_unit - 1) / p.kb_unit;
+    if (p.split_k > U) { p.split_k = U; if (p.s_long > U) p.s_long = U; }
+    const int ss = p.split_k - p.s_long;
+    int at = 0;
+    for (int z = 0; z < p.split_k; ++z) {
+      p.unit_begin[z] = at;
+      if (ss == 0) at += U / p.split_k + (z < U % p.split_k ? 1 : 0);
+      else if (z < p.s_long) at += best_x;
+      else {
+        const int y_total = U - p.s_long * best_x, zs = z - p.s_long;
+        at += y_total / ss + (zs < y_total % ss ? 1 : 0);
+      }
+    }
+    p.unit_begin[p.split_k] = U;
+    for (int z = p.split_k + 1; z <= kTcMaxSlices; ++z) p.unit_begin[z] = U;
   }
   p.ctrl_bytes = p.gather == kOptCoop
                      ? round_up((kCoopCtrlInts + static_cast<size_t>(groups) *
@@ -227,11 +295,10 @@ int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& map
   // persistent launch: never more workers than are resident at once, each loops over its tiles
   p.tiles_x = static_cast<int>(tile_grid.x);
   p.tiles_y = static_cast<int>(tile_grid.y);
-  p.tiles_z = static_cast<int>(tile_grid.z);
   const long long n_tiles = static_cast<long long>(tile_grid.x) * tile_grid.y * tile_grid.z;
   // (cooperative gather: every SM takes part in the gather, also those without a tile)
-  const int workers = n_tiles < max_workers[dev] && GATHER != kGatherCoop ? static_cast<int>(n_tiles)
-                                                                          : max_workers[dev];
+  const int workers = n_tiles < max_workers[dev] && GATHER != kGatherCoop && p.s_long == p.split_k
+                          ? static_cast<int>(n_tiles) : max_workers[dev];
   cfg.gridDim = dim3(static_cast<unsigned>(PAIR ? 2 * workers : workers));
   {
     ProfileScope prof(GRASS_K_PROJECT_TC, s);
@@ -393,7 +460,10 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   p.r = r;
   p.k_blocks = plan.k_blocks;
   p.split_k = plan.split_k;
+  p.s_long = plan.s_long;
   p.kb_unit = plan.kb_unit;
+  p.groups = count;
+  for (int z = 0; z <= kTcMaxSlices; ++z) p.unit_begin[z] = static_cast<unsigned short>(plan.unit_begin[z]);
   p.status = status;
   p.norm_part = fused_norms ? part[0] : nullptr;
   const bool in_kernel = plan.gather == kOptCta || plan.gather == kOptCoop;
@@ -407,11 +477,14 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   p.m = static_cast<int>(m);
   p.r_pad = plan.r_pad;
   p.coop_ctrl = nullptr;
+  p.coop_warps = opts.gather_warps > 0 ? opts.gather_warps : 8;
   p.coop_chunks = static_cast<int>((T + kCoopChunk - 1) / kCoopChunk);
   p.coop_cg = (plan.r_pad + kCoopCols - 1) / kCoopCols;
-  {
-    const int n_units = (plan.k_blocks + plan.kb_unit - 1) / plan.kb_unit;
-    p.coop_pmax = n_units / plan.split_k + (n_units % plan.split_k != 0 ? 1 : 0);
+  p.coop_pmax_long = p.coop_pmax_short = 0;
+  for (int z = 0; z < plan.split_k; ++z) {
+    const int units = plan.unit_begin[z + 1] - plan.unit_begin[z];
+    int& pm = z < plan.s_long ? p.coop_pmax_long : p.coop_pmax_short;
+    if (units > pm) pm = units;
   }
   if (plan.gather == kOptCoop) {
     // queue head and per-chunk counters start at zero for every launch
@@ -434,6 +507,7 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   // tile space handed to the persistent kernel (x counts pairs of CTAs in pair mode)
   dim3 grid(static_cast<unsigned>(plan.pair ? plan.n_blocks / 2 : plan.n_blocks),
             static_cast<unsigned>(plan.r_blocks), static_cast<unsigned>(plan.split_k * count));
+  if (plan.unit_begin[plan.split_k] > 65535) return GRASS_ERR_UNSUPPORTED;   // 16-bit slice table
   const int kernel_gather = plan.gather == kOptCta ? kGatherCta
                             : plan.gather == kOptCoop ? kGatherCoop : kGatherNone;
   const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, kernel_gather, grid, plan.smem_bytes,
@@ -481,6 +555,8 @@ void describe_plan(const TcPlan& plan, int count, grass_project_plan_t* out) {
   out->ctas_per_slice = plan.n_blocks * plan.r_blocks * count;
   out->cta_pair = plan.pair ? 1 : 0;
   out->token_slices = plan.split_k;
+  out->short_slices = plan.split_k - plan.s_long;
+  out->long_slice_tokens = (plan.unit_begin[1] - plan.unit_begin[0]) * plan.kb_unit * plan.bk;
   out->tokens_per_stage = plan.bk;
   out->stages = plan.stages;
   out->workspace_bytes = plan_ws_bytes(plan, count) + 256;

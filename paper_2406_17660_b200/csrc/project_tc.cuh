@@ -89,6 +89,7 @@ __host__ __device__ constexpr int tc_stages(int MB, int A_SLABS) {
 }
 
 constexpr int kTcMaxGroup = 8;
+constexpr int kTcMaxSlices = 64;    // token slices per layer
 
 constexpr int kGatherNone = 0, kGatherCta = 1, kGatherCoop = 2;
 // Cooperative gather: tokens per chunk (one readiness counter each), columns per item, and the
@@ -108,11 +109,14 @@ struct TcMaps {
 struct TcParams {
   int T, n, r;          // logical sizes
   int k_blocks;         // ceil(T / tokens per stage)
-  int split_k;          // token slices per layer
-  int kb_unit;          // slices start on multiples of this many token blocks
-  int tiles_x, tiles_y, tiles_z;   // tile space: n-tiles (per pair if PAIR), row blocks,
-                                   // layers * split_k
-  // Up to kTcMaxGroup same-shaped layers share one launch: blockIdx.z = group * split_k + split.
+  int split_k;          // token slices per layer; slice z covers the units
+                        // [unit_begin[z], unit_begin[z + 1]) of kb_unit token blocks each
+  int s_long;           // the first s_long slices are "long", the others "short" (see the
+                        // tile schedule in the kernel); s_long == split_k: all alike
+  int kb_unit;
+  unsigned short unit_begin[kTcMaxSlices + 1];
+  int tiles_x, tiles_y; // output tiles of one layer: n-tiles (per pair if PAIR), row blocks
+  int groups;           // up to kTcMaxGroup same-shaped layers share one launch
   float* out[kTcMaxGroup];        // split_k == 1: Gc, else partials [split][r][ld_out]
   long long ld_out;     // row pitch of out, elements
   long long split_stride;  // elements between partials of consecutive splits
@@ -128,7 +132,8 @@ struct TcParams {
   int* coop_ctrl;
   int coop_chunks;      // chunks per layer = ceil(T / kCoopChunk)
   int coop_cg;          // column groups = ceil(r_pad / kCoopCols)
-  int coop_pmax;        // most chunks in one token slice
+  int coop_pmax_long, coop_pmax_short;   // most chunks in one long / short token slice
+  int coop_warps;       // gather warps per CTA that take part (1..8)
   float* norm_part;     // non-NULL: row-norm mode.  Nothing of D is stored; instead
                         // norm_part[g * ld_norm + j] = sum of D[j, c]^2 over the 32 columns c of group g
   long long ld_norm;
@@ -157,7 +162,7 @@ template <int NI>
 __device__ __forceinline__ void coop_gather_part(const unsigned short* __restrict__ src,
                                                  long long lddy, unsigned short* __restrict__ dst,
                                                  int r_pad, int col0, const int (&rows)[8], int tok0,
-                                                 int T, int lane) {
+                                                 int T, int lane, int* publish) {
   constexpr int TU = (32 / NI) < (kCoopChunk / kCoopParts) ? (32 / NI) : (kCoopChunk / kCoopParts);   // tokens per batch of loads
   constexpr int NTOK = kCoopChunk / kCoopParts;           // tokens of this part
   // Every load is unconditional (rows and tokens clamped to valid ones, the value discarded at
@@ -175,6 +180,13 @@ __device__ __forceinline__ void coop_gather_part(const unsigned short* __restric
       const unsigned short* line = src + static_cast<long long>(tok < T ? tok : T - 1) * lddy;
 #pragma unroll
       for (int i = 0; i < NI; ++i) v[u][i] = ptx::ld_nc_na_u16(line + safe[i]);
+    }
+    if (publish != nullptr) {
+      // the previous item's stores (all lanes, program order + warp barrier) become visible
+      // before its counter moves; the fence's wait hides behind the loads just issued
+      __syncwarp();
+      if (lane == 0) ptx::flag_arrive_release(publish);
+      publish = nullptr;
     }
 #pragma unroll
     for (int u = 0; u < TU; ++u) {
@@ -223,22 +235,40 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                               ~static_cast<uintptr_t>(1023));
   const int rank = PAIR ? static_cast<int>(ptx::cluster_ctarank()) : 0;
-  // Persistent workers: a worker (a CTA, or a CTA pair) takes the tiles w, w + W, w + 2W, ... of
-  // the linear tile space [tile_x fastest, then row block, then (layer, token slice)], i.e. the
-  // same order a plain grid would be dispatched in, so concurrent workers still sweep the tokens
-  // together.  The grid never exceeds what is resident at once: the whole grid is dispatched
-  // immediately and kernels of other streams can be scheduled beside it.
+  // Persistent workers and the tile schedule.  A tile is (n-tile bx, row block by, layer, token
+  // slice z); a worker is a CTA, or a CTA pair.  With W workers and N tiles of equal length the
+  // last wave is only partly filled whenever W does not divide N.  The host therefore cuts
+  // the tokens into s_long long slices and (optionally) a few short ones: the long tiles are
+  // dealt round-robin (worker w takes w, w + W, ...: the order a plain grid would be dispatched
+  // in, so concurrent workers sweep the tokens together and share operands through L2), and the
+  // R = N_long mod W workers that got one long tile more than the others are done; the other
+  // W - R workers share the short tiles round-robin.  The slice lengths are chosen so that both
+  // kinds of worker finish together.  Every tile writes its own split-K partial, so the
+  // result does not depend on which worker ran it.
   const int n_workers = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
   const int worker = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
-  const int n_tiles = p.tiles_x * p.tiles_y * p.tiles_z;
-  // token slices in units of kb_unit blocks: u_per or u_per + 1 units each
-  const int n_units = (p.k_blocks + p.kb_unit - 1) / p.kb_unit;
-  const int u_per = n_units / p.split_k, u_rem = n_units % p.split_k;
+  const int txy = p.tiles_x * p.tiles_y;
+  const int s_short = p.split_k - p.s_long;
+  const int n_long = txy * p.groups * p.s_long, n_short = txy * p.groups * s_short;
+  const int sched_R = n_long % n_workers;
+  const int short_workers = sched_R > 0 ? n_workers - sched_R : n_workers;
+  const int my_long = worker < n_long ? (n_long - worker + n_workers - 1) / n_workers : 0;
 
-  // decode a linear tile index (identical in every role)
+  // the k-th tile of this worker (identical in every role); false when there is none
   struct Tile { int c_base, r0, grp, z, kb_begin, kb_count; };
-  auto decode = [&](int L) {
-    Tile t;
+  auto sched = [&](int k, Tile& t) -> bool {
+    int L, sl, z0;
+    if (k < my_long) {
+      L = worker + k * n_workers;
+      sl = p.s_long;
+      z0 = 0;
+    } else {
+      if (sched_R > 0 && worker < sched_R) return false;
+      L = (sched_R > 0 ? worker - sched_R : worker) + (k - my_long) * short_workers;
+      if (L >= n_short) return false;
+      sl = s_short;
+      z0 = p.s_long;
+    }
     const int bx = L % p.tiles_x;
     const int rest = L / p.tiles_x;
     const int by = rest % p.tiles_y, bz = rest / p.tiles_y;
@@ -246,12 +276,13 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     // pair_base + (mb * 2 + rank) * 128; otherwise the CTA owns MB consecutive blocks.
     t.c_base = PAIR ? bx * (2 * MB * 128) + rank * 128 : bx * (MB * 128);
     t.r0 = by * R_CTA;
-    t.grp = bz / p.split_k;                 // which layer of the group
-    t.z = bz - t.grp * p.split_k;           // which token slice
-    t.kb_begin = (t.z * u_per + (t.z < u_rem ? t.z : u_rem)) * p.kb_unit;
-    t.kb_count = (u_per + (t.z < u_rem ? 1 : 0)) * p.kb_unit;
-    if (t.kb_begin + t.kb_count > p.k_blocks) t.kb_count = p.k_blocks - t.kb_begin;
-    return t;
+    t.grp = bz / sl;                        // which layer of the group
+    t.z = z0 + bz - t.grp * sl;             // which token slice
+    t.kb_begin = static_cast<int>(p.unit_begin[t.z]) * p.kb_unit;
+    int kb_end = static_cast<int>(p.unit_begin[t.z + 1]) * p.kb_unit;
+    if (kb_end > p.k_blocks) kb_end = p.k_blocks;
+    t.kb_count = kb_end - t.kb_begin;
+    return true;
   };
 
   if (threadIdx.x == 0) {
@@ -289,8 +320,9 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     int s = 0, issued = 0;
     uint32_t ph = 0;
     bool alive = true;
-    for (int L = worker; L < n_tiles && alive; L += n_workers) {
-      const Tile t = decode(L);
+    for (int k = 0; alive; ++k) {
+      Tile t;
+      if (!sched(k, t)) break;
       const CUtensorMap* map = is_x ? &maps.x[t.grp] : &maps.a[t.grp];
       int xcoord;
       if (is_x) {
@@ -382,8 +414,9 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
       int s = 0;
       uint32_t ph = 0, tile_ph = 0;
       bool first_tile = true;
-      for (int L = worker; L < n_tiles && ok; L += n_workers) {
-        const Tile t = decode(L);
+      for (int k = 0; ok; ++k) {
+        Tile t;
+        if (!sched(k, t)) break;
         if (!first_tile) {
           // the accumulators are reused: the epilogue warps (of both CTAs) must have read the
           // previous tile out of TMEM before the first MMA of this one overwrites it
@@ -437,42 +470,74 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
         tile_ph ^= 1u;
       }
     }
-  } else if (COOP && warp >= kTcThreads / 32) {
+  } else if (COOP && warp >= kTcThreads / 32 && warp - kTcThreads / 32 < p.coop_warps) {
     // ================= gather warps (COOP): shared queue over the whole launch =================
     // Item = (token slice bz, chunk position pp in the slice, column group, part): one warp
     // copies dY[t, idx[j]] for the part's 16 tokens and up to 256 columns j into Ag[t, j].
     // Queue order follows the GEMM: slices grouped by the wave of tiles that first touches them,
     // inside a group chunk position first, so every running tile finds its next chunk early.
     // Padding items (a slice shorter than coop_pmax) are skipped.
-    const int txy = p.tiles_x * p.tiles_y;
-    const int n_waves = (n_tiles + n_workers - 1) / n_workers;
+    // Slices are taken in the order the schedule above starts them: the slices of each full
+    // wave of long tiles, then one last group holding the slices first touched by the partly
+    // filled long wave together with ALL short slices (the workers without a tile in that wave
+    // start on the short tiles at the same moment).  Inside a group the chunk position runs
+    // slowest, so every running tile finds its next chunk early.
     const int per_chunk = p.coop_cg * kCoopParts;
-    const int per_slice = p.coop_pmax * per_chunk;
-    const int total = p.tiles_z * per_slice;
+    const int full_waves = n_long / n_workers;
+    const int bz_full = full_waves > 0 ? (full_waves * n_workers - 1) / txy + 1 : 0;  // slices of full waves
+    const int cnt_long_last = p.groups * p.s_long - bz_full;      // long slices left for the last group
+    const int cnt_last = cnt_long_last + p.groups * s_short;
+    const int pmax_last = cnt_long_last > 0 && p.coop_pmax_long > p.coop_pmax_short ? p.coop_pmax_long
+                                                                                    : p.coop_pmax_short;
+    const int items_full = bz_full * p.coop_pmax_long * per_chunk;
+    const int total = items_full + cnt_last * pmax_last * per_chunk;
+    // The counter of a finished item is published from inside the next item (after its first
+    // loads are issued), so that the fence's round trip does not sit between two batches of
+    // loads.  (Popping the next item ahead of time as well was slower: an item popped early sits
+    // idle while its chunk's other parts complete, and the consumers wait for the last part.)
+    int* publish = nullptr;
     while (true) {
       int q = 0;
       if (lane == 0) q = atomicAdd(p.coop_ctrl, 1);
       q = __shfl_sync(0xffffffffu, q, 0);
       if (q >= total) break;
-      int bz_lo = 0, bz_hi = 0, base = 0;
-      for (int w = 0; w < n_waves; ++w) {
-        const int last_tile = ((w + 1) * n_workers < n_tiles ? (w + 1) * n_workers : n_tiles) - 1;
-        bz_hi = last_tile / txy + 1;
-        const int items = (bz_hi - bz_lo) * per_slice;
-        if (q < base + items || w == n_waves - 1) break;
-        base += items;
-        bz_lo = bz_hi;
+      int pp, z, grp, rem2;
+      if (q < items_full) {
+        // which full wave: its new slices are [bz_lo, bz_hi)
+        int bz_lo = 0, bz_hi = 0, base = 0;
+        for (int w = 0; w < full_waves; ++w) {
+          bz_hi = ((w + 1) * n_workers - 1) / txy + 1;
+          const int items = (bz_hi - bz_lo) * p.coop_pmax_long * per_chunk;
+          if (q < base + items) break;
+          base += items;
+          bz_lo = bz_hi;
+        }
+        const int in_wave = q - base, cnt = bz_hi - bz_lo;
+        pp = in_wave / (cnt * per_chunk);
+        const int rem = in_wave - pp * (cnt * per_chunk);
+        const int bz = bz_lo + rem / per_chunk;
+        rem2 = rem - (rem / per_chunk) * per_chunk;
+        grp = bz / p.s_long;
+        z = bz - grp * p.s_long;
+      } else {
+        const int in_wave = q - items_full;
+        pp = in_wave / (cnt_last * per_chunk);
+        const int rem = in_wave - pp * (cnt_last * per_chunk);
+        const int si = rem / per_chunk;
+        rem2 = rem - si * per_chunk;
+        if (si < cnt_long_last) {
+          const int bz = bz_full + si;
+          grp = bz / p.s_long;
+          z = bz - grp * p.s_long;
+        } else {
+          const int bzs = si - cnt_long_last;
+          grp = bzs / s_short;
+          z = p.s_long + bzs - grp * s_short;
+        }
       }
-      const int in_wave = q - base, cnt = bz_hi - bz_lo;
-      const int pp = in_wave / (cnt * per_chunk);
-      const int rem = in_wave - pp * (cnt * per_chunk);
-      const int bz = bz_lo + rem / per_chunk;
-      const int rem2 = rem - (rem / per_chunk) * per_chunk;
       const int cg = rem2 / kCoopParts, part = rem2 - cg * kCoopParts;
-      const int grp = bz / p.split_k, z = bz - grp * p.split_k;
-      const int units = u_per + (z < u_rem ? 1 : 0);
-      if (pp >= units || bz >= p.tiles_z) continue;          // padding item
-      const int chunk = z * u_per + (z < u_rem ? z : u_rem) + pp;   // kb_unit blocks = one chunk
+      const int chunk = static_cast<int>(p.unit_begin[z]) + pp;    // kb_unit blocks = one chunk
+      if (chunk >= static_cast<int>(p.unit_begin[z + 1])) continue;   // padding item
       const int col0 = cg * kCoopCols;
       const int32_t* idx = p.idx[grp];
       int rows[8];
@@ -493,12 +558,14 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
       unsigned short* dst = reinterpret_cast<unsigned short*>(p.Ag[grp]);
       const int tok0 = chunk * kCoopChunk + part;
       const int cols = p.r_pad - col0;
-      if (cols <= 64) coop_gather_part<2>(src, p.lddy, dst, p.r_pad, col0, rows, tok0, p.T, lane);
-      else if (cols <= 128) coop_gather_part<4>(src, p.lddy, dst, p.r_pad, col0, rows, tok0, p.T, lane);
-      else coop_gather_part<8>(src, p.lddy, dst, p.r_pad, col0, rows, tok0, p.T, lane);
-      __threadfence();           // this lane's stores are performed device-wide ...
+      if (cols <= 64) coop_gather_part<2>(src, p.lddy, dst, p.r_pad, col0, rows, tok0, p.T, lane, publish);
+      else if (cols <= 128) coop_gather_part<4>(src, p.lddy, dst, p.r_pad, col0, rows, tok0, p.T, lane, publish);
+      else coop_gather_part<8>(src, p.lddy, dst, p.r_pad, col0, rows, tok0, p.T, lane, publish);
+      publish = p.coop_ctrl + kCoopCtrlInts + grp * p.coop_chunks + chunk;
+    }
+    if (publish != nullptr) {
       __syncwarp();
-      if (lane == 0) ptx::flag_arrive_release(p.coop_ctrl + kCoopCtrlInts + grp * p.coop_chunks + chunk);
+      if (lane == 0) ptx::flag_arrive_release(publish);
     }
   } else if (FUSED && warp >= kTcThreads / 32) {
     // ================= gather warps (FUSED): dY[t, idx[j]] -> swizzled B-operand slabs =================
@@ -511,8 +578,9 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     int s = 0;
     uint32_t ph = 0;
     bool alive = true;
-    for (int L = worker; L < n_tiles && alive; L += n_workers) {
-      const Tile t = decode(L);
+    for (int k = 0; alive; ++k) {
+      Tile t;
+      if (!sched(k, t)) break;
       const unsigned short* src = reinterpret_cast<const unsigned short*>(p.dY[t.grp]);
       const int32_t* idx = p.idx[t.grp];
       int rows[A_SLABS][2];
@@ -594,8 +662,9 @@ project_tc_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     const int half = (warp - 2) >> 2;   // which of the quarter's two warps
     uint32_t tile_ph = 0;
     bool alive = true;
-    for (int L = worker; L < n_tiles && alive; L += n_workers) {
-      const Tile t = decode(L);
+    for (int k = 0; alive; ++k) {
+      Tile t;
+      if (!sched(k, t)) break;
       // one polling lane per warp, with back-off: this wait lasts a whole main loop
       int got = 1;
       if (lane == 0) {
