@@ -201,15 +201,16 @@ def nr_scores(norms, method, seed, layer_id, epoch):
     smallest t -- equivalently the r largest scores w_k / (-log u_k) -- are
     distributed exactly as r successive draws without replacement.
     u_k = (word_k + 1/2) * 2^-32, word_k = Philox word (k mod 4) of block
-    (k div 4, layer_id, epoch, tag).  The score is rounded to fp32 and the
-    decision is taken on those fp32 values (ties to the lower row).
+    (k div 4, layer_id, epoch, tag).  Scores are fp64 and ranked as such (ties to
+    the lower row); an implementation that ranks rounded scores may differ only
+    where two scores at the selection threshold agree to its rounding.
     """
     lam = _check_norms(norms)
     m = lam.shape[0]
     w = sampling_weights(lam, method)
     words = draw_words(m, seed, layer_id, epoch).astype(np.float64)
     u = (words + 0.5) * 2.0 ** -32
-    return (w / -np.log(u)).astype(np.float32)
+    return w / -np.log(u)
 
 
 def select_without_replacement(norms, r, method, seed, layer_id, epoch):
