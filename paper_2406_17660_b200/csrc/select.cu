@@ -291,17 +291,26 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
   __shared__ int s_cbase[kWarps];
   // local[k] = running sum inside the segment (warp scan per 32 rows, carried across the
   // segment); cdf[k] = base[warp] + local[k] with base[w + 1] = base[w] + local total of w added
-  // by one thread in order, so the running sum is exactly monotone across segment borders and a
-  // draw can never land on a zero-weight row.
+  // by one thread in order.  A shuffle scan adds the same terms in a different order in every
+  // lane, so neighbouring entries can disagree in the last bit; what a draw must never do is
+  // land on a row of zero weight (rho would be infinite).  Therefore a zero-weight row takes
+  // the entry of the nearest row of positive weight before it, bit for bit (0 if the slice has
+  // none, which makes it equal to the previous slice's last entry): cdf[k] > target can then
+  // first become true only at a row of positive weight.
   auto slice_scan = [&](int k0) {
     const int k = k0 + lane;
-    double v = k < k_end ? sampling_weight(a.method, nrm[k]) : 0.0;
+    const double w = k < k_end ? sampling_weight(a.method, nrm[k]) : 0.0;
+    double v = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const double up = __shfl_up_sync(0xffffffffu, v, o);
       if (lane >= o) v += up;
     }
-    return v;
+    const uint32_t positive = __ballot_sync(0xffffffffu, w > 0.0);
+    const uint32_t at_or_before = positive & (0xffffffffu >> (31 - lane));
+    const int src = at_or_before != 0u ? 31 - __clz(at_or_before) : 0;
+    const double taken = __shfl_sync(0xffffffffu, v, src);
+    return at_or_before != 0u ? taken : 0.0;
   };
   {
     double run = 0.0;
@@ -351,6 +360,9 @@ __global__ void __launch_bounds__(kThreads) select_kernel(SelectArgs a) {
       const int mid = (lo + hi) >> 1;
       if (cdf[mid] > target) hi = mid; else lo = mid + 1;
     }
+    // (the entries of zero-weight rows repeat their predecessor's, so lo has positive weight;
+    // the loop below only guards the very last rows when the target rounds up to the total)
+    while (lo > 0 && !(sampling_weight(a.method, nrm[lo]) > 0.0)) --lo;
     atomicAdd(&counts[lo], 1);
   }
   __syncthreads();

@@ -184,6 +184,29 @@ def test_select_without_replacement(method, m, r):
         assert np.all(np.abs(sc[swapped] - thr) <= 1e-6 * thr), "mismatch beyond the near-tie allowance"
 
 
+@pytest.mark.parametrize("method", [grass.SEL_MULTINOMIAL_NORM, grass.SEL_MULTINOMIAL_NORM2])
+def test_sampling_never_lands_on_a_zero_weight_row(method):
+    """Many rows of zero weight between rows of very different weight: the fp64 running sum of a
+    warp scan is not exactly monotone there, and a draw that landed on a zero-weight row would
+    make rho infinite.  The kernel's running sum repeats the predecessor's entry on such rows."""
+    rng = np.random.default_rng(77)
+    for trial in range(4):
+        m, r = 13824, 1024
+        lam = np.exp(3.0 * rng.standard_normal(m)).astype(np.float32)
+        lam[rng.random(m) < 0.6] = 0.0
+        status, idx, rho = _gpu_select(lam, r, method, seed=trial, layer_id=trial, epoch=trial)
+        assert status == 0
+        assert np.all(lam[idx] > 0) and np.all(np.isfinite(rho)) and np.all(rho > 0)
+        sigma, rho_ref = oracle.select(lam, r, method, seed=trial, layer_id=trial, epoch=trial)
+        if np.array_equal(idx, sigma):
+            np.testing.assert_allclose(rho, rho_ref, rtol=1e-6)
+        else:
+            c = np.cumsum(oracle.sampling_weights(lam.astype(np.float64), method))
+            u = oracle.draw_words(r, trial, trial, trial).astype(np.float64) * 2.0 ** -32 * c[-1]
+            gap = np.min(np.abs(c[None, :] - u[:, None]), axis=1) / c[-1]
+            assert np.sum(idx != sigma) <= np.sum(gap < 1e-6)
+
+
 def test_select_without_replacement_needs_enough_positive_rows():
     lam = np.zeros(64, dtype=np.float32)
     lam[:5] = 1.0
@@ -255,9 +278,9 @@ def _assert_close_gc(got, want, tol=1e-4):
 @pytest.mark.parametrize("T,m,n,r", [(512, 256, 256, 32), (100, 50, 70, 7), (33, 65, 129, 65)])
 def test_project_fp32(T, m, n, r):
     got, want = _project_case(T, m, n, r, torch.float32, seed=T + r, dup=(r == 7))
-    assert rel_fro(got, want) <= 1e-5
+    _assert_close_gc(got, want, 1e-5)
     got, want = _project_case(T, m, n, r, torch.float32, seed=T, identity=True, with_rho=False)
-    assert rel_fro(got, want) <= 1e-5
+    _assert_close_gc(got, want, 1e-5)
 
 
 @pytest.mark.parametrize("T,m,n,r,ldx,kw", [
@@ -282,10 +305,8 @@ def test_project_fp32(T, m, n, r):
 ])
 def test_project_bf16_tensor_core(T, m, n, r, ldx, kw):
     got, want = _project_case(T, m, n, r, torch.bfloat16, seed=T + n + r, ldx=ldx, **kw)
-    assert np.all(np.isfinite(got))
-    err = rel_fro(got, want)
-    assert err <= 1e-2                                    # acceptance tolerance
-    assert err <= 1e-4, err                               # what fp32 accumulation must deliver
+    assert rel_fro(got, want) <= 1e-2                     # acceptance tolerance
+    _assert_close_gc(got, want, 1e-4)                     # what fp32 accumulation must deliver
 
 
 def test_project_bf16_is_bit_reproducible_and_flags_bad_rows():
@@ -383,19 +404,46 @@ def _run_layer(m, n, T, r, dtype, method, K, steps, alpha, reset, seed, layer_id
                        w_is_bf16=(dtype == torch.bfloat16), trace=trace)
     for t, (dY, X) in enumerate(batches):
         before = layer.W.clone()
+        M_prev, V_prev = f64(layer.M), f64(layer.V)
         layer.step(dY.to(DEV), X.to(DEV))
         grass.grass_device_status()
         ref = trace[t]
         assert np.array_equal(layer.idx.cpu().numpy(), ref["sigma"]), f"step {t}: rows differ"
         np.testing.assert_allclose(layer.rho.cpu().numpy(), ref["rho"], rtol=2e-5)
         tol = 1e-5 if dtype == torch.float32 else 1e-4
-        assert rel_fro(f64(layer.Gc), ref["Gc"]) <= tol
+        _assert_close_gc(f64(layer.Gc), ref["Gc"], tol)
+        # Adam and the apply step from the GPU's own G_C and previous state: this isolates the
+        # update kernels from the GEMM's summation order, so the stated 1e-5 applies element-wise
+        if reset and t % K == 0:
+            M_prev[:] = 0.0
+            V_prev[:] = 0.0
+        g_gpu = f64(layer.Gc)
+        M1, V1, U1 = oracle.adam_update(M_prev, V_prev, g_gpu, lr, b1, b2, eps, layer.adam_step)
+        scale_M = b1 * np.abs(M_prev) + (1 - b1) * np.abs(g_gpu)
+        assert np.all(np.abs(f64(layer.M) - M1) <= 1e-5 * scale_M + 1e-30), f"step {t}: M"
+        np.testing.assert_allclose(f64(layer.V), V1, rtol=1e-5, atol=1e-30)
+        s = layer.adam_step
+        scale_U = lr * (scale_M / (1 - b1 ** s)) / (np.sqrt(V1 / (1 - b2 ** s)) + eps)
+        assert np.all(np.abs(f64(layer.U) - U1) <= 1e-5 * scale_U + 1e-30), f"step {t}: U"
+        sigma, rho_gpu = ref["sigma"], layer.rho.cpu().numpy()
+        touched = np.unique(sigma)
+        untouched = np.setdiff1d(np.arange(m), sigma)
+        got = f64(layer.W)
+        assert torch.equal(layer.W[untouched], before[untouched])      # bit-identical
+        exact = oracle.scatter_update(f64(before), f64(layer.U), sigma, rho_gpu, alpha)[touched]
+        if dtype == torch.float32:
+            np.testing.assert_allclose(got[touched], exact, rtol=1e-5, atol=1e-9)
+        else:
+            want = oracle.round_to_bf16(exact)
+            ulp = np.ldexp(1.0, np.floor(np.log2(np.maximum(np.abs(exact), 2.0 ** -126))).astype(int) - 7)
+            diff = np.abs(got[touched] - want)
+            assert np.all(diff <= ulp * 1.0001), f"step {t}: W off by more than one bf16 ulp"
+            assert np.mean(diff > 0) < 0.01                             # rounding-boundary cases only
+        # end to end against the oracle's own trajectory (secondary: the bf16 GEMM's fp32
+        # summation order feeds into these)
         assert rel_fro(f64(layer.M), ref["M"]) <= tol
         assert rel_fro(f64(layer.V), ref["V"]) <= 2 * tol
         assert rel_fro(f64(layer.U), ref["U"]) <= 10 * tol
-        untouched = np.setdiff1d(np.arange(m), ref["sigma"])
-        got = f64(layer.W)
-        assert torch.equal(layer.W[untouched], before[untouched])      # bit-identical
         if dtype == torch.float32:
             np.testing.assert_allclose(got, ref["W"], rtol=1e-5, atol=1e-8)
         else:
@@ -414,6 +462,14 @@ def test_layer_steps_bf16_multinomial_with_refresh():
     """60M-shaped q projection at reduced T: multinomial-norm, rho, refresh at t = 0 and 2."""
     _run_layer(512, 512, 2048, 128, torch.bfloat16, grass.SEL_MULTINOMIAL_NORM, K=2, steps=4,
                alpha=0.25, reset=False, seed=3, layer_id=5)
+
+
+@pytest.mark.parametrize("m,n", [(1024, 1024), (1024, 2736)], ids=["350m_q", "350m_down"])
+def test_layer_steps_350m_topr_ten_steps_across_a_refresh(m, n):
+    """LLaMA-350M q and down shapes, top-r, r = 256, K = 5, ten steps (refresh at t = 0 and 5,
+    state reset on), at a token count the oracle affords; every step is checked element-wise."""
+    _run_layer(m, n, 4096, 256, torch.bfloat16, grass.SEL_TOPR, K=5, steps=10, alpha=0.25,
+               reset=True, seed=6, layer_id=1)
 
 
 def test_layer_steps_bf16_topr_reset():
@@ -555,7 +611,7 @@ def test_batched_projection_and_update_match_the_oracle_layer_by_layer(count, T,
     grass.grass_device_status()
     for g in range(count):
         want = oracle.project_grad(f64(dYs[g]), f64(Xs[g]), sig[g], rho[g])
-        assert rel_fro(f64(Gc[g]), want) <= 1e-4, g
+        _assert_close_gc(f64(Gc[g]), want, 1e-4)
         # the update against the single-layer call on the same projected gradient: bit-identical
         M1 = torch.zeros_like(M[g]); V1 = torch.zeros_like(V[g]); W1 = Ws[g].to(DEV).clone()
         grass.grass_adam_scatter(Gc[g], M1, V1, None, W1, idx[g], rhod[g], 1e-3, 0.9, 0.999, 1e-8, 1, 0.25)
