@@ -4,6 +4,10 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--rank r]
     python bench.py --impl reference ...      # the fp64 CPU oracle, timed on the host cores
 
+--gpus N (N > 1) runs N independent replicas, one process per GPU: under a launcher
+(torch.distributed.run sets WORLD_SIZE) this process is one of them; without one it starts
+them itself.
+
 A step is one iteration of the paper's Algorithm 1 over every layer of the
 workload: on a refresh iteration (t = 0 mod K) the dense gradient, its row
 norms and the selection, then for every layer projected gradient, Adam and
@@ -29,12 +33,11 @@ if ROOT not in sys.path:
 METRIC = "TFLOP/s per layer-step (select+project+Adam+scatter)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel.  ncu captured
-# one n = 4096 layer (339.1 MB: X and the gathered operand each read once, see
-# profiles/project_tc_kernel_llama7b_q_r1024.md); traffic grows in proportion to the layers and
-# to 2Tn + 2Tr, so the three batched launches of a step move 4 x 339 MB (q,k,v,o), 2 x 339 MB
-# (gate, up) and about 792 MB (down): 942 MB per launch on average.  None where nothing was captured.
-NCU_TRAFFIC_BYTES = {"llama7b_block_r1024": 942e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu
+# capture of the default workload at T = 8192 scaled by 4 to T = 32768 (every operand is streamed
+# once per launch, so traffic grows in proportion to the tokens), averaged over the three
+# launches of a step.  None where nothing was captured.
+NCU_TRAFFIC_BYTES = {}
 
 
 def load_peaks():
@@ -224,7 +227,8 @@ def aggregate_max(local_ms: float, dist_mod=None) -> float:
     return float(t.item())
 
 
-def run_gpu(args):
+def measure_workload(ctx, name, r, steps, warmup, want_e2e, want_cpu, args):
+    """Run one workload on this rank's GPU and return its result line (rank 0; None elsewhere)."""
     import torch
     import torch.distributed as dist
     import paper_2406_17660_b200 as grass
@@ -232,38 +236,27 @@ def run_gpu(args):
     from paper_2406_17660_b200 import workloads
     from paper_2406_17660_b200.step import GrassLayer, GrassLayerGroup, GrassWorkspace
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
-    torch.cuda.set_device(local_rank)
-    dev = f"cuda:{local_rank}"
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device(dev))
-    grass.load_library()
-    peaks = load_peaks()
-
-    wl = workloads.get(args.workload, r=args.rank, T=args.tokens, layers=args.layers)
+    world, rank, local_rank, dev, peaks = (ctx["world"], ctx["rank"], ctx["local_rank"], ctx["dev"],
+                                           ctx["peaks"])
+    wl = workloads.get(name, r=r, T=args.tokens, layers=args.layers)
     K = args.refresh_every or wl.K
     # ---- inputs: one block of distinct tensors, shared by all blocks (replicas are independent:
     # every rank holds its own full copy of the workload, no data-path collective) ----
     block_in = []
-    for pi, (name, m, n) in enumerate(wl.shapes):
+    for pi, (pname, m, n) in enumerate(wl.shapes):
         dY = syn.make_dY(wl.T, m, wl.dtype, proj=pi, device=dev, ld=syn.pad_to(m, 8))
         X = syn.make_X(wl.T, n, wl.dtype, proj=pi, device=dev, ld=syn.pad_to(n, 8))
         block_in.append((dY, X))
     # Layers are independent, so consecutive layers go to alternating streams (each with its own
-    # scratch): the HBM-bound kernels of one layer (column gather, Adam, apply) then run beside
-    # the tensor-bound GEMM of its neighbour.  --streams 1 puts everything on one stream.
+    # scratch): the HBM-bound kernels of one layer (Adam, apply, split-K reduce) then run beside
+    # the GEMM of its neighbour.  --streams 1 puts everything on one stream.
     n_streams = max(1, args.streams)
     main_stream = torch.cuda.current_stream()
     streams = [main_stream] + [torch.cuda.Stream() for _ in range(n_streams - 1)]
     wss = [GrassWorkspace([(m, n) for _, m, n in wl.shapes], wl.T, wl.r, wl.dtype, wl.method,
                           device=dev) for _ in range(n_streams)]
     layers = []
-    for i, (li, pi, name, m, n) in enumerate(wl.layer_list()):
+    for i, (li, pi, pname, m, n) in enumerate(wl.layer_list()):
         W = syn.make_W(m, n, wl.dtype, layer=li, proj=pi, device=dev, ld=syn.pad_to(n, 8))
         layer = GrassLayer(W, min(wl.r, m), wl.method, K, wl.alpha, wl.lr, wl.beta1, wl.beta2,
                            wl.eps, reset_state=wl.reset_state, seed=0,
@@ -289,9 +282,8 @@ def run_gpu(args):
                                                                       device=dev)
         units.append({"obj": obj, "pis": [pi for pi, _ in members], "layers": [l for _, l in members]})
         i = j
-    # Within a step the units are independent, so their order is free.  The first unit's column
-    # gather and the last unit's update have nothing to hide behind: start with the unit that
-    # gathers the fewest bytes (layers x m) and keep the rest in block order.
+    # Within a step the units are independent, so their order is free: start with the unit whose
+    # dY is smallest (layers x m) and keep the rest in block order.
     if len(units) > 2:
         first = min(range(len(units)), key=lambda u: len(units[u]["layers"]) * units[u]["layers"][0].m)
         units.insert(0, units.pop(first))
@@ -328,43 +320,46 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(warmup, 3)):
         one_step()
     grass.grass_device_status()
 
     # ---- pass A: the timed region ----
     rewind()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.1)
     barrier()
     ev[0].record()
-    for i in range(args.steps):
+    for i in range(steps):
         one_step()
         ev[i + 1].record()
     barrier()
     total_ms = aggregate_max(ev[0].elapsed_time(ev[-1]), dist if world > 1 else None)
-    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
     grass.grass_device_status()
 
     # ---- pass B: the same steps with every kernel launch bracketed by events ----
     rewind()
-    n_refresh = (args.steps + K - 1) // K
-    cap = args.steps * len(layers) * 5 + n_refresh * len(layers) * 8 + 16
+    n_refresh = (steps + K - 1) // K
+    cap = steps * len(layers) * 5 + n_refresh * len(layers) * 8 + 16
     # one stream for this pass: an event pair must bracket one kernel running alone, not a kernel
     # sharing the GPU with another layer's kernels
     single_stream[0] = True
     grass.grass_profile_begin(cap)
-    for i in range(args.steps):
+    for i in range(steps):
         one_step()
     launches, recs = grass.grass_profile_end()
     single_stream[0] = False
     clocks = sampler.stop() if rank == 0 else None
+    if args.launch_log:
+        with open(args.launch_log, "w") as f:
+            json.dump([(kname, round(1e3 * ms, 2)) for kname, ms in recs], f)
     per_kernel = {}
-    for name, ms in recs:
-        k = per_kernel.setdefault(name, {"launches": 0, "ms": 0.0})
+    for kname, ms in recs:
+        k = per_kernel.setdefault(kname, {"launches": 0, "ms": 0.0})
         k["launches"] += 1
         k["ms"] += ms
     prof_total = sum(k["ms"] for k in per_kernel.values())
@@ -372,21 +367,38 @@ def run_gpu(args):
         k["share"] = k["ms"] / prof_total if prof_total > 0 else 0.0
         k["avg_us"] = 1e3 * k["ms"] / k["launches"]
 
-    refresh_steps = [i for i in range(args.steps) if i % K == 0]
-    regular_steps = [i for i in range(args.steps) if i % K != 0]
-    flops_total = wl.flops_regular() * args.steps + wl.flops_refresh_extra() * len(refresh_steps)
+    refresh_steps = [i for i in range(steps) if i % K == 0]
+    regular_steps = [i for i in range(steps) if i % K != 0]
+    flops_total = wl.flops_regular() * steps + wl.flops_refresh_extra() * len(refresh_steps)
     value = world * flops_total / (total_ms * 1e-3) / 1e12
     n_layers = len(layers)
 
-    # ---- roofline of the dominant kernel (tcgen05 projection GEMM) ----
+    # ---- roofline of the dominant kernel (tcgen05 projection GEMM, which now also gathers) ----
+    # The measured peak that applies depends on how long the GPU has been under load: a timed
+    # region of well under a second runs at burst clocks, a long one settles at the power cap.
     roofline = None
+    region_s = (total_ms + prof_total) * 1e-3
     if "project_tc" in per_kernel:
         tc = per_kernel["project_tc"]
         achieved = flops_total / (tc["ms"] * 1e-3) / 1e12
-        peak = peaks["bf16_tflops_sustained"]
+        burst, sustained = peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
+        use_burst = region_s < 1.0
+        peak = burst if use_burst else sustained
+        path_ms = sum(per_kernel[k]["ms"] for k in ("gather", "project_tc", "splitk_reduce")
+                      if k in per_kernel)
         roofline = {"kernel": "project_tc_kernel", "bound": "tensor", "achieved": achieved,
                     "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                    "peak_source": f"{peaks['source']} cuBLAS bf16, sustained",
+                    "peak_source": f"{peaks['source']} cuBLAS bf16, "
+                                   f"{'burst' if use_burst else 'sustained'} "
+                                   f"(timed region {region_s:.2f} s)",
+                    "frac_of_burst_peak": achieved / burst,
+                    "frac_of_sustained_peak": achieved / sustained,
+                    # the projection as the method sees it: selected-column gather (inside the GEMM
+                    # kernel unless a pre-pass was asked for) + GEMM + split-K reduce, same flops
+                    "path": {"kernels": [k for k in ("gather", "project_tc", "splitk_reduce")
+                                         if k in per_kernel],
+                             "ms": path_ms, "achieved": flops_total / (path_ms * 1e-3) / 1e12,
+                             "frac": flops_total / (path_ms * 1e-3) / 1e12 / peak},
                     "traffic": NCU_TRAFFIC_BYTES.get(f"{wl.name}_r{wl.r}")}
     elif "project_fp32" in per_kernel:
         pk = per_kernel["project_fp32"]
@@ -400,22 +412,29 @@ def run_gpu(args):
         rn = sum(min(wl.r, m) * n for _, m, n in wl.shapes) * wl.layers
         wbytes = 2 if wl.dtype == torch.bfloat16 else 4
         if "adam" in per_kernel:
-            b = 24.0 * rn * args.steps
+            b = 24.0 * rn * steps
             hbm["adam"] = {"gbs": b / (per_kernel["adam"]["ms"] * 1e-3) / 1e9}
         if "scatter" in per_kernel:
-            b = (4.0 + 2 * wbytes) * rn * args.steps
+            b = (4.0 + 2 * wbytes) * rn * steps
             hbm["scatter"] = {"gbs": b / (per_kernel["scatter"]["ms"] * 1e-3) / 1e9}
         if "adam_scatter" in per_kernel:
-            b = (20.0 + 2 * wbytes) * rn * args.steps      # g, M, V in; M, V out; W in and out
+            b = (20.0 + 2 * wbytes) * rn * steps      # g, M, V in; M, V out; W in and out
             hbm["adam_scatter"] = {"gbs": b / (per_kernel["adam_scatter"]["ms"] * 1e-3) / 1e9}
-        # (the step takes its row norms from the GEMM epilogue; the stand-alone row-norm kernel's
-        # bandwidth is measured by profile_case, see profiles/)
+        if "gather" in per_kernel:
+            # a pre-pass (only when asked for): algorithmic bytes 2Tr in + 2Tr out per layer; what
+            # it must touch is every 128-byte line of dY that holds a selected column, and the copy
+            alg = sum(4.0 * wl.T * min(wl.r, m) for _, m, n in wl.shapes) * wl.layers * steps
+            touched = sum(2.0 * wl.T * m * (1.0 - (1.0 - min(wl.r, m) / m) ** 64) +
+                          2.0 * wl.T * min(wl.r, m) for _, m, n in wl.shapes) * wl.layers * steps
+            sec = per_kernel["gather"]["ms"] * 1e-3
+            hbm["gather"] = {"gbs": alg / sec / 1e9, "touched_gbs": touched / sec / 1e9,
+                             "algorithmic_bytes": alg, "touched_bytes": touched}
         for v in hbm.values():
             v["frac_of_hbm_peak"] = v["gbs"] / peaks["hbm_gbs"]
 
     # ---- e2e: host buffers in, host result out, through the same public calls ----
     e2e = None
-    if not args.no_e2e:
+    if want_e2e:
         host_in = []
         for dY, X in block_in:
             hd = torch.empty(dY.shape, dtype=dY.dtype, pin_memory=True)
@@ -423,13 +442,14 @@ def run_gpu(args):
             hd.copy_(dY)
             hx.copy_(X)
             host_in.append((hd, hx))
+
         def like(t):      # same shape AND row pitch (empty_like would drop the padding)
             return torch.empty((t.shape[0], t.stride(0)), dtype=t.dtype, device=t.device)[:, : t.shape[1]]
 
         stage = [(like(d), like(x)) for d, x in block_in]
         max_rn = max(l.Gc.numel() for _, l in layers)
         host_out = [torch.empty(max_rn, dtype=torch.float32, pin_memory=True) for _ in wl.shapes]
-        e2e_steps = min(args.steps, args.e2e_steps)
+        e2e_steps = min(steps, args.e2e_steps)
         h2d = sum(d.numel() * d.element_size() + x.numel() * x.element_size()
                   for d, x in host_in) * wl.layers
         d2h = sum(l.Gc.numel() * 4 for _, l in layers)
@@ -471,22 +491,23 @@ def run_gpu(args):
 
     # ---- the oracle on the host cores, rank 0 of a single-GPU run only ----
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and want_cpu:
         T_gen = min(wl.T, 16384)            # about 10 s of oracle work on 16 host threads
         ins = [(syn.to_f32_numpy(d[:T_gen]), syn.to_f32_numpy(x[:T_gen])) for d, x in block_in]
         Ws = [syn.to_f32_numpy(layers[pi][1].W) for pi in range(len(wl.shapes))]
-        sub = workloads.get(args.workload, r=args.rank, T=T_gen, layers=args.layers)
+        sub = workloads.get(name, r=r, T=T_gen, layers=args.layers)
         res = time_oracle(sub, ins, Ws, budget_s=args.cpu_budget, steps=1, warmup=0)
         res["sample"] = res["sample"].replace(f"of {T_gen} tokens", f"of {wl.T} tokens")
         cpu_baseline = {"value": res["value"], "unit": "TFLOP/s", "cores": blas_threads(),
                         "kind": "oracle", "sample": res["sample"], "seconds": res["seconds"]}
 
+    line = None
     if rank == 0:
         reg_ms = statistics.mean(step_ms[i] for i in regular_steps) if regular_steps else None
         ref_ms = statistics.mean(step_ms[i] for i in refresh_steps) if refresh_steps else None
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world,
-            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
+            "steps": steps, "warmup": max(warmup, 3), "ms_per_step": total_ms / steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if wl.dtype == torch.bfloat16 else "f32", "data": "synthetic",
             "config": {"workload": wl.name, "layers": n_layers, "T": wl.T, "r": wl.r,
@@ -501,9 +522,81 @@ def run_gpu(args):
             "us_per_layer_step_refresh": None if ref_ms is None else 1e3 * ref_ms / n_layers,
             "tflops_regular_steps": None if reg_ms is None else wl.flops_regular() / (reg_ms * 1e-3) / 1e12,
             "roofline": roofline, "hbm_kernels": hbm, "kernels": per_kernel,
-            "profiled_pass_ms_per_step": prof_total / args.steps,
+            "profiled_pass_ms_per_step": prof_total / steps,
             "gpu_launches": launches, "e2e": e2e, "cpu_baseline": cpu_baseline, "clocks": clocks,
         }
+    # release this workload's device memory before the next one is built
+    del block_in, layers, units, wss
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    return line
+
+
+def replica_command(args, argv):
+    """The command that runs `--gpus N` as N replicas, one process per GPU (argv: this
+    process's own arguments)."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+            f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1", "--master-port", str(port),
+            os.path.abspath(__file__)] + list(argv)
+
+
+def check_launch(args):
+    """--check-launch: every rank joins a CPU (gloo) process group and rank 0 reports how many
+    ranks the launch produced; touches no GPU."""
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    count = 1
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo")
+        t = torch.ones(1, dtype=torch.float64)
+        dist.all_reduce(t)
+        count = int(t.item())
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"check_launch": True, "n_gpus": args.gpus, "ranks": count}))
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2406_17660_b200 as grass
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    grass.load_library()
+    ctx = {"world": world, "rank": rank, "local_rank": local_rank, "dev": dev, "peaks": load_peaks()}
+
+    line = measure_workload(ctx, args.workload, args.rank, args.steps, args.warmup,
+                            not args.no_e2e, not args.no_cpu_baseline, args)
+    # The other half of the target configuration (LLaMA-13B shapes, and r = 256), as short runs
+    # with their own clock records; only beside the default workload.
+    also = []
+    if not args.no_also and args.workload == "llama7b_block" and args.rank is None and \
+            args.tokens is None and args.layers is None:
+        for name, r in (("llama13b_block", None), ("llama7b_block", 256), ("llama13b_block", 256)):
+            sub = measure_workload(ctx, name, r, min(args.steps, 20), 3, False, False, args)
+            if sub is not None:
+                also.append({k: sub[k] for k in ("value", "unit", "steps", "ms_per_step", "config",
+                                                 "us_per_layer_step_regular", "us_per_layer_step_refresh",
+                                                 "tflops_regular_steps", "roofline", "hbm_kernels",
+                                                 "kernels", "clocks")})
+    if rank == 0:
+        line["also"] = also
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -526,10 +619,21 @@ def main():
     ap.add_argument("--no-batched", dest="batched", action="store_false",
                     help="one set of launches per layer instead of per run of same-shaped layers")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
+    ap.add_argument("--launch-log", default=None,
+                    help="write (kernel, microseconds) of every launch of the profiled pass to this file")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-also", action="store_true",
+                    help="skip the short extra runs (13B shapes, r = 256) beside the default workload")
+    ap.add_argument("--check-launch", action="store_true",
+                    help="only report how many ranks --gpus N produced (CPU, no GPU work)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    # --gpus N without a launcher: start N replicas ourselves, one process per GPU
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(subprocess.call(replica_command(args, sys.argv[1:])))
+    if args.check_launch:
+        check_launch(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

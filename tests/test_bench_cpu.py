@@ -59,3 +59,23 @@ def test_workload_table_matches_the_configs():
     w = workloads.get("config1")
     assert w.dtype == torch.float32 and w.alpha == 1.0 and w.K == 1
     assert workloads.get("llama1b", r=64).r == 64
+
+
+def test_gpus_flag_starts_that_many_replicas_by_itself():
+    """`bench.py --gpus 2` with no launcher around it re-executes itself under
+    torch.distributed.run as two ranks (checked on CPU: the ranks only join a gloo group)."""
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--check-launch"]
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["ranks"] == 2 and lines[0]["n_gpus"] == 2
+    sys.path.insert(0, ROOT)
+    import bench
+
+    class A:
+        gpus = 4
+    argv = bench.replica_command(A, ["--gpus", "4", "--steps", "3"])
+    assert "--nproc-per-node=4" in argv and argv[-4:] == ["--gpus", "4", "--steps", "3"]
+    assert "127.0.0.1" in argv
