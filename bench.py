@@ -34,10 +34,12 @@ METRIC = "TFLOP/s per layer-step (select+project+Adam+scatter)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu
-# capture of the default workload at T = 8192 scaled by 4 to T = 32768 (every operand is streamed
-# once per launch, so traffic grows in proportion to the tokens), averaged over the three
-# launches of a step.  None where nothing was captured.
-NCU_TRAFFIC_BYTES = {}
+# capture of the default workload at T = 8192 (1717.6 MB over the three GEMM launches of a step)
+# scaled by 4 to T = 32768 (every operand is streamed once per launch, so traffic grows in
+# proportion to the tokens), averaged over the three launches.  The kernel gathers the selected
+# dY columns itself, so this includes every 128-byte line of dY that holds one.  None where
+# nothing was captured.
+NCU_TRAFFIC_BYTES = {"llama7b_block_r1024": 2290e6}
 
 
 def load_peaks():

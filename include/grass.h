@@ -114,10 +114,15 @@ int grass_select(const float* norms, int64_t m, int32_t r, int method, uint64_t 
  * pooling allocator already owns the whole device, so that a raw cudaMalloc
  * would fail; a plugin that is handed tensors but no allocator; a step on a
  * latency-critical path where the device-wide synchronisation an allocation
- * implies is not acceptable.  The scratch (the fp64 running sum and the
- * per-row hit counters) lives in a fixed array inside the library image:
+ * implies is not acceptable.  The scratch (room for the fp64 running sum and
+ * the per-row hit counters) lives in a fixed array inside the library image:
  * GRASS_SELECT_STATIC_MAX_M rows, 12 bytes each (192 KiB), held by every GPU
- * that loads the library until the process exits.
+ * that loads the library until the process exits.  How much of it a call
+ * touches: the kernel stages the hit counters in shared memory for every m this
+ * call accepts, and the running sum too while m <= 12800, so only the
+ * running-sum part of the array is ever used, and only by the sampling methods
+ * with replacement at 12800 < m <= 16384 (the 13824-row LLaMA-13B projections);
+ * all other calls leave the array alone.
  *   - m > GRASS_SELECT_STATIC_MAX_M returns GRASS_ERR_WORKSPACE (and says so on
  *     stderr); nothing is launched.  All other arguments and errors are as for
  *     grass_select.

@@ -239,6 +239,8 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 }
 
 // bf16 matrix [rows][cols] with row pitch ld (elements): box = {64 cols, bk rows}, 128B swizzle.
+// Encoded on every call: a host-side cache keyed by (pointer, shape, pitch) was measured and
+// saved nothing (40.8 us against 41.9 us of host time per batched call of four 60M layers).
 bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int bk) {
   PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
   if (fn == nullptr) return false;

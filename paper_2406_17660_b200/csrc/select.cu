@@ -549,8 +549,9 @@ extern "C" int grass_select_static(const float* norms, int64_t m, int32_t r, int
   a.epoch = epoch;
   a.idx = idx;
   a.rho = rho;
-  // The kernel writes every running-sum entry it later reads and zeroes the
-  // m hit counters before counting, so whatever an earlier call left in the
-  // array is never observed.
+  // Of the array the kernel can reach only the running sum, and only for m > 12800 with a
+  // with-replacement method (everything else is staged in shared memory); it writes every
+  // running-sum entry before reading it, so whatever an earlier call left there is never
+  // observed.
   return launch_select(a, static_cast<cudaStream_t>(stream));
 }
