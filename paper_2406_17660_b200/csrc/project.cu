@@ -76,6 +76,11 @@ int choose_gather(bool has_idx, const PlanOpts& opts, int r_cta, int tiles_x, in
   if (opts.gather == kOptCoop) return kOptCoop;
   if (opts.gather == kOptAuto && cta_ok && tiles_x <= 2 && static_cast<int64_t>(r) * 12 >= m)
     return kOptCta;
+  // Few selected rows (r <= 128): the GEMM is a pure HBM stream of X and the gather is as large
+  // as the GEMM itself; as two kernels the gather of one layer overlaps the GEMM of another
+  // stream's layer, which measured better than one kernel doing both (1B shapes, r = 64 / 128:
+  // 98 / 116 us per layer-step against 107 / 128).
+  if (opts.gather == kOptAuto && cta_ok) return kOptPrepass;
   return kOptCoop;
 }
 
