@@ -382,26 +382,62 @@ def measure_workload(ctx, name, r, steps, warmup, want_e2e, want_cpu, args):
     region_s = (total_ms + prof_total) * 1e-3
     if "project_tc" in per_kernel:
         tc = per_kernel["project_tc"]
-        achieved = flops_total / (tc["ms"] * 1e-3) / 1e12
         burst, sustained = peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
         use_burst = region_s < 1.0
-        peak = burst if use_burst else sustained
+        tpeak = burst if use_burst else sustained
+        which = "burst" if use_burst else "sustained"
         path_ms = sum(per_kernel[k]["ms"] for k in ("gather", "project_tc", "splitk_reduce")
                       if k in per_kernel)
-        roofline = {"kernel": "project_tc_kernel", "bound": "tensor", "achieved": achieved,
-                    "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                    "peak_source": f"{peaks['source']} cuBLAS bf16, "
-                                   f"{'burst' if use_burst else 'sustained'} "
-                                   f"(timed region {region_s:.2f} s)",
-                    "frac_of_burst_peak": achieved / burst,
-                    "frac_of_sustained_peak": achieved / sustained,
+        # algorithmic bytes of the projection per layer-step: X once, the r selected columns of
+        # dY once, G_C out (2Tn + 2Tr + 4rn); per refresh: X and dY once (2Tn + 2Tm).  What the
+        # memory system cannot avoid touching is larger: every 128-byte line of dY that holds a
+        # selected column (measured with ncu), i.e. 2Tm (1 - (1 - r/m)^64) instead of 2Tr.
+        rs = [(min(wl.r, m), m, n) for _, m, n in wl.shapes]
+        alg_reg = sum(2.0 * wl.T * n + 2.0 * wl.T * r_ + 4.0 * r_ * n for r_, m, n in rs) * wl.layers
+        touched_reg = sum(2.0 * wl.T * n + 2.0 * wl.T * m * (1.0 - (1.0 - r_ / m) ** 64) + 4.0 * r_ * n
+                          for r_, m, n in rs) * wl.layers
+        dense = sum(2.0 * wl.T * n + 2.0 * wl.T * m for r_, m, n in rs) * wl.layers
+        # the launches of the regular steps only: the dense GEMMs of refresh iterations are the
+        # same kernel on all m rows and are accounted separately ("dense" below)
+        alg_total = alg_reg * steps
+        touched_total = touched_reg * steps
+        flops_proj = wl.flops_regular() * steps
+        t_tensor = wl.flops_regular() / (tpeak * 1e12)
+        t_hbm = alg_reg / (peaks["hbm_gbs"] * 1e9)
+        tensor_side = {"achieved": flops_proj / (tc["ms"] * 1e-3) / 1e12, "unit": "TFLOP/s", "peak": tpeak,
+                       "peak_source": f"{peaks['source']} cuBLAS bf16, {which} (timed region {region_s:.2f} s)"}
+        tensor_side["frac"] = tensor_side["achieved"] / tpeak
+        hbm_side = {"achieved": alg_total / (tc["ms"] * 1e-3) / 1e9, "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                    "peak_source": f"{peaks['source']} HBM copy bandwidth",
+                    "touched_gbs": touched_total / (tc["ms"] * 1e-3) / 1e9}
+        hbm_side["frac"] = hbm_side["achieved"] / peaks["hbm_gbs"]
+        hbm_side["frac_touched"] = hbm_side["touched_gbs"] / peaks["hbm_gbs"]
+        bound = "hbm" if t_hbm > t_tensor else "tensor"
+        main_side = hbm_side if bound == "hbm" else tensor_side
+        roofline = {"kernel": "project_tc_kernel", "bound": bound,
+                    "bound_rule": "regular step: algorithmic bytes / HBM peak vs flops / tensor peak, "
+                                  f"{1e6 * t_hbm:.0f} us vs {1e6 * t_tensor:.0f} us",
+                    "achieved": main_side["achieved"], "peak": main_side["peak"],
+                    "unit": main_side["unit"], "frac": main_side["frac"],
+                    "peak_source": main_side["peak_source"],
+                    "tensor": tensor_side, "hbm": hbm_side,
+                    "frac_of_burst_peak": tensor_side["achieved"] / burst,
+                    "frac_of_sustained_peak": tensor_side["achieved"] / sustained,
                     # the projection as the method sees it: selected-column gather (inside the GEMM
-                    # kernel unless a pre-pass was asked for) + GEMM + split-K reduce, same flops
+                    # kernel unless a pre-pass is used) + GEMM + split-K reduce, same flops
                     "path": {"kernels": [k for k in ("gather", "project_tc", "splitk_reduce")
                                          if k in per_kernel],
-                             "ms": path_ms, "achieved": flops_total / (path_ms * 1e-3) / 1e12,
-                             "frac": flops_total / (path_ms * 1e-3) / 1e12 / peak},
+                             "ms": path_ms, "achieved": flops_proj / (path_ms * 1e-3) / 1e12,
+                             "frac": flops_proj / (path_ms * 1e-3) / 1e12 / tpeak,
+                             "hbm_frac_touched": touched_total / (path_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
                     "traffic": NCU_TRAFFIC_BYTES.get(f"{wl.name}_r{wl.r}")}
+        if "project_tc_dense" in per_kernel and refresh_steps:
+            dn = per_kernel["project_tc_dense"]
+            ach = wl.flops_refresh_extra() * len(refresh_steps) / (dn["ms"] * 1e-3) / 1e12
+            roofline["dense"] = {"what": "refresh iterations: dY^T X on all m rows with the row-norm "
+                                         "epilogue, 2mTn flop per layer", "bound": "tensor",
+                                 "achieved": ach, "unit": "TFLOP/s", "peak": tpeak, "frac": ach / tpeak,
+                                 "algorithmic_bytes": dense * len(refresh_steps)}
     elif "project_fp32" in per_kernel:
         pk = per_kernel["project_fp32"]
         achieved = flops_total / (pk["ms"] * 1e-3) / 1e12

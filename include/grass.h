@@ -373,12 +373,14 @@ typedef enum {
   GRASS_K_ROW_NORMS = 0,
   GRASS_K_SELECT = 1,
   GRASS_K_GATHER = 2,        /* copy of the selected dY columns */
-  GRASS_K_PROJECT_TC = 3,    /* tcgen05 projection GEMM */
+  GRASS_K_PROJECT_TC = 3,    /* tcgen05 projection GEMM on the r selected rows */
   GRASS_K_SPLITK_REDUCE = 4,
   GRASS_K_PROJECT_FP32 = 5,
   GRASS_K_ADAM = 6,
   GRASS_K_SCATTER = 7,
-  GRASS_K_ADAM_SCATTER = 8   /* fused Adam + apply */
+  GRASS_K_ADAM_SCATTER = 8,  /* fused Adam + apply */
+  GRASS_K_PROJECT_TC_DENSE = 9  /* the same GEMM kernel on all m rows (idx = NULL): dense gradient
+                                   or its row norms, i.e. the launches of a refresh iteration */
 } grass_kernel_t;
 int grass_profile_begin(int32_t max_launches);
 int grass_profile_end(int32_t* kernel_id, float* ms, int32_t* n_launches);

@@ -66,7 +66,7 @@ _SIGNATURES = {
 }
 
 KERNEL_NAMES = ["row_norms", "select", "gather", "project_tc", "splitk_reduce", "project_fp32",
-                "adam", "scatter", "adam_scatter"]
+                "adam", "scatter", "adam_scatter", "project_tc_dense"]
 
 
 def load_library():

@@ -264,7 +264,8 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
 }
 
 template <int MB, int NSLAB, bool PAIR, int GATHER>
-int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& maps, TcParams p) {
+int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& maps, TcParams p,
+                  int kernel_id) {
   constexpr bool FUSED = GATHER != kGatherNone;   // the variants with eight extra warps
   static bool attr_set[64] = {false};
   static int max_workers[64] = {0};
@@ -308,7 +309,7 @@ int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& map
                           ? static_cast<int>(n_tiles) : max_workers[dev];
   cfg.gridDim = dim3(static_cast<unsigned>(PAIR ? 2 * workers : workers));
   {
-    ProfileScope prof(GRASS_K_PROJECT_TC, s);
+    ProfileScope prof(kernel_id, s);
     GRASS_CUDA_TRY(cudaLaunchKernelEx(&cfg, project_tc_kernel<MB, NSLAB, PAIR, GATHER>, maps, p));
   }
   return GRASS_OK;
@@ -317,10 +318,10 @@ int launch_tc_one(dim3 tile_grid, size_t smem, cudaStream_t s, const TcMaps& map
 // (MB, NSLAB) with MB * 64 * NSLAB <= 512 TMEM columns; pairs need an even NSLAB.
 // gather: kGatherNone / kGatherCta (tiles of at most 128 rows) / kGatherCoop.
 int launch_tc(int MB, int nslab, bool pair, int gather, dim3 grid, size_t smem, cudaStream_t s,
-              const TcMaps& maps, const TcParams& p) {
+              const TcMaps& maps, const TcParams& p, int kernel_id) {
 #define GRASS_TC_CASE(mb, ns, pr, ga)                                                          \
   if (MB == mb && nslab == ns && pair == pr && gather == ga)                                   \
-    return launch_tc_one<mb, ns, pr, ga>(grid, smem, s, maps, p)
+    return launch_tc_one<mb, ns, pr, ga>(grid, smem, s, maps, p, kernel_id)
 #define GRASS_TC_BOTH(mb, ns, pr)                                                              \
   GRASS_TC_CASE(mb, ns, pr, kGatherNone);                                                      \
   GRASS_TC_CASE(mb, ns, pr, kGatherCoop)
@@ -518,7 +519,7 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   const int kernel_gather = plan.gather == kOptCta ? kGatherCta
                             : plan.gather == kOptCoop ? kGatherCoop : kGatherNone;
   const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, kernel_gather, grid, plan.smem_bytes,
-                           s, maps, p);
+                           s, maps, p, gather ? GRASS_K_PROJECT_TC : GRASS_K_PROJECT_TC_DENSE);
   if (rc != GRASS_OK) return rc;
   if (norms != nullptr) {
     ProfileScope prof(GRASS_K_ROW_NORMS, s);
