@@ -160,6 +160,8 @@ int grass_select_static(const float* norms, int64_t m, int32_t r, int method, ui
  * accepts any alignment.  The sum over tokens is split into a fixed number of
  * slices added in a fixed order: results are bit-reproducible run to run.
  * A row index outside [0, m) contributes zeros and sets the status word.
+ * GRASS_BF16: T <= 2 097 120 tokens (GRASS_ERR_UNSUPPORTED beyond: token slices are
+ * kept in a 16-bit table of 32- to 128-token units).
  */
 size_t grass_project_workspace_bytes(int64_t T, int64_t m, int64_t n, int32_t r, int dt);
 int grass_project_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx, int dt,

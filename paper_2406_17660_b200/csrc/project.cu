@@ -415,6 +415,7 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
                                        : make_plan(T, m, n, r, gather, opts, false, count);
   if (plan.gather == kOptPrepass && T > 65535LL * kGatherTokens)
     return GRASS_ERR_UNSUPPORTED;                                            // pre-pass grid.y
+  if (plan.unit_begin[plan.split_k] > 65535) return GRASS_ERR_UNSUPPORTED;   // 16-bit slice table
   const bool fused_norms = norms != nullptr && plan.split_k == 1;
   const size_t per_layer = fused_norms ? norm_part_bytes(m, n) : plan.ag_bytes + plan.part_bytes;
   const size_t need = plan.ctrl_bytes + per_layer * count;
@@ -515,7 +516,7 @@ int project_bf16(int count, const void* const* dY, int64_t lddy, const void* con
   // tile space handed to the persistent kernel (x counts pairs of CTAs in pair mode)
   dim3 grid(static_cast<unsigned>(plan.pair ? plan.n_blocks / 2 : plan.n_blocks),
             static_cast<unsigned>(plan.r_blocks), static_cast<unsigned>(plan.split_k * count));
-  if (plan.unit_begin[plan.split_k] > 65535) return GRASS_ERR_UNSUPPORTED;   // 16-bit slice table
+
   const int kernel_gather = plan.gather == kOptCta ? kGatherCta
                             : plan.gather == kOptCoop ? kGatherCoop : kGatherNone;
   const int rc = launch_tc(plan.MB, plan.r_cta / 64, plan.pair, kernel_gather, grid, plan.smem_bytes,

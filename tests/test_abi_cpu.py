@@ -77,6 +77,31 @@ def test_argument_errors_are_returned_without_a_device(lib):
     assert lib.grass_scatter_update(fake, 5, 8, 8, 8, fake, 8, fake, null, 4, 0.25, null) == 3
 
 
+def test_projection_options_and_limits_are_checked_on_the_host(lib):
+    null = ctypes.c_void_p(None)
+    fake = ctypes.c_void_p(0x1000)
+    # more tokens than the 16-bit slice table can describe: rejected before anything is launched
+    assert lib.grass_project_grad(fake, 1000, fake, 8, 1, 2 ** 31 - 1, 1000, 8, fake, null, 4, fake, 8,
+                                  fake, 1 << 40, null) == 3
+    # options out of range
+    plan = binding.ProjectPlan()
+    for bad in (dict(gather=4), dict(n_blocks_per_cta=3), dict(cta_pair=3), dict(token_slices=-1),
+                dict(gather_warps=9)):
+        opts = binding.ProjectOpts(**bad)
+        assert lib.grass_project_plan(1, 1024, 512, 512, 128, ctypes.byref(opts), ctypes.byref(plan)) == 1
+    # the plan query is host-only and honours explicit options
+    p = binding.grass_project_plan(1, 4096, 2048, 1024, 512, dict(gather=binding.GATHER_PREPASS, token_slices=3))
+    assert p["gather"] == binding.GATHER_PREPASS and p["token_slices"] == 3 and p["short_slices"] == 0
+    assert p["rows_per_tile"] == 512 and p["workspace_bytes"] >= 4096 * 512 * 2 + 3 * 512 * 1024 * 4
+    p = binding.grass_project_plan(1, 4096, 2048, 1024, 512, dict(gather=binding.GATHER_COOPERATIVE))
+    assert p["gather"] == binding.GATHER_COOPERATIVE
+    assert binding.grass_project_plan(1, 4096, 2048, 1024, 512)["gather"] == binding.GATHER_COOPERATIVE
+    assert binding.grass_project_plan(4, 65536, 512, 512, 128)["gather"] == binding.GATHER_IN_CTA
+    # in-CTA gather is only for tiles of at most 128 rows: the request falls back to the default
+    assert binding.grass_project_plan(1, 4096, 2048, 1024, 512, dict(gather=binding.GATHER_IN_CTA))["gather"] \
+        == binding.GATHER_COOPERATIVE
+
+
 def test_workspace_queries_are_host_only_and_monotone(lib):
     assert binding.grass_select_workspace_bytes(4096, 256, binding.SEL_TOPR) >= 256
     a = binding.grass_select_workspace_bytes(4096, 256, binding.SEL_MULTINOMIAL_NORM)
