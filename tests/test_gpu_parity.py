@@ -681,6 +681,10 @@ def test_cooperative_gather_over_token_slices(T, m, n, r, slices):
     opts = dict(gather=grass.GATHER_COOPERATIVE, token_slices=slices)
     got, want = _project_case(T, m, n, r, torch.bfloat16, seed=T + r + slices, opts=opts)
     _assert_close_gc(got, want)
+    # fewer gather warps per CTA: same items, same bits
+    opts["gather_warps"] = 1 + slices % 4
+    again, _ = _project_case(T, m, n, r, torch.bfloat16, seed=T + r + slices, opts=opts)
+    assert np.array_equal(again, got)
 
 
 def test_cooperative_gather_is_bit_reproducible_and_matches_the_prepass():
