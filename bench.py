@@ -58,7 +58,7 @@ def load_peaks():
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_power_cap,clocks.mem,clocks.max.mem")
     NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index: int):
@@ -86,7 +86,7 @@ class ClockSampler:
             self.proc.kill()
         self.file.flush()
         self.file.seek(0)
-        sm, mx, reasons, power = [], [], set(), []
+        sm, mx, reasons, power, mem, mem_mx = [], [], set(), [], [], []
         for line in self.file:
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 7:
@@ -97,6 +97,11 @@ class ClockSampler:
                 power.append(float(parts[2]))
             except ValueError:
                 continue
+            try:
+                mem.append(float(parts[7]))
+                mem_mx.append(float(parts[8]))
+            except (ValueError, IndexError):
+                pass
             for name, val in zip(self.NAMES, parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
@@ -105,6 +110,8 @@ class ClockSampler:
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
                        samples=len(sm), power_w_max=max(power))
+            if mem:
+                out.update(mem_mhz=statistics.median(mem), mem_max_mhz=max(mem_mx))
         return out
 
 
