@@ -111,3 +111,34 @@ def test_workspace_queries_are_host_only_and_monotone(lib):
     assert 1024 * 128 * 2 <= small < big
     assert big >= 32768 * 1024 * 2
     assert binding.grass_project_workspace_bytes(1024, 512, 512, 128, binding.F32) >= 256
+
+
+def test_plans_are_sane_over_a_sweep_of_shapes(lib):
+    """The host plan (tile rows, n-blocks per CTA, pairs, long and short token slices, gather
+    mode) for every benchmark shape and a grid of odd ones: structural invariants only."""
+    shapes = [(c, T, m, n, r) for c in (1, 2, 4) for T in (31, 512, 4100, 32768, 65536)
+              for m, n in ((512, 512), (1376, 512), (2048, 5461), (4096, 4096), (11008, 4096),
+                           (4096, 11008), (13824, 5120), (300, 328))
+              for r in (1, 64, 100, 256, 600, 1024) if r <= m]
+    seen_modes = set()
+    for c, T, m, n, r in shapes:
+        p = binding.grass_project_plan(c, T, m, n, r)
+        assert p["rows_per_tile"] % 64 == 0 and p["rows_per_tile"] * p["row_blocks"] >= r
+        assert p["rows_per_tile"] * p["n_blocks_per_cta"] <= 512          # TMEM columns
+        assert p["n_blocks_per_cta"] in (1, 2, 4) and p["cta_pair"] in (0, 1)
+        assert not p["cta_pair"] or p["rows_per_tile"] % 128 == 0
+        assert 1 <= p["token_slices"] <= 64 and 0 <= p["short_slices"] <= 3
+        assert p["short_slices"] < p["token_slices"]
+        assert 0 < p["long_slice_tokens"] <= T + 127
+        assert p["gather"] in (binding.GATHER_PREPASS, binding.GATHER_IN_CTA, binding.GATHER_COOPERATIVE)
+        if p["gather"] == binding.GATHER_IN_CTA:
+            assert p["rows_per_tile"] <= 128
+        if p["gather"] == binding.GATHER_COOPERATIVE:
+            assert p["long_slice_tokens"] % 128 == 0 or p["token_slices"] == 1
+        gathered = 0 if p["gather"] == binding.GATHER_IN_CTA else T * p["rows_per_tile"] * p["row_blocks"] * 2 * c
+        partials = p["token_slices"] * r * n * 4 * c if p["token_slices"] > 1 else 0
+        assert p["workspace_bytes"] >= gathered + partials
+        slack = p["token_slices"] * r * 3 * 4 * c + 4 * c * (T // 128 + 1) + 1024 * c + 1024   # pitch, counters, alignment
+        assert p["workspace_bytes"] <= gathered + partials + slack
+        seen_modes.add(p["gather"])
+    assert len(seen_modes) == 3
