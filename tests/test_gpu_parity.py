@@ -687,6 +687,38 @@ def test_cooperative_gather_over_token_slices(T, m, n, r, slices):
     assert np.array_equal(again, got)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_projection_on_random_small_shapes_all_gather_modes(seed):
+    """Seeded random shapes (ragged T, m, n, r; repeated rows; with and without rho; 1..3 layers)
+    through every gather mode and the plain call; every result against the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    for _ in range(6):
+        T = int(rng.integers(1, 700))
+        m = int(rng.integers(1, 900))
+        n = int(rng.integers(1, 600))
+        r = int(rng.integers(1, m + 1))
+        count = int(rng.integers(1, 4))
+        ldx, lddy = syn.pad_to(n, 8), syn.pad_to(m, 8)
+        Xs = [syn.make_X(T, n, torch.bfloat16, seed0=seed, proj=g) for g in range(count)]
+        dYs = [syn.make_dY(T, m, torch.bfloat16, seed0=seed, proj=g) for g in range(count)]
+        Xd = [syn._padded(t.to(DEV), ldx) for t in Xs]
+        dYd = [syn._padded(t.to(DEV), lddy) for t in dYs]
+        sig = [np.sort(rng.choice(m, r, replace=bool(rng.integers(0, 2)))) for _ in range(count)]
+        rho = [(0.5 + rng.random(r)).astype(np.float32) for _ in range(count)]
+        idx = [torch.tensor(x, dtype=torch.int32, device=DEV) for x in sig]
+        rhod = [torch.tensor(x, device=DEV) for x in rho]
+        want = [oracle.project_grad(f64(dYs[g]), f64(Xs[g]), sig[g], rho[g]) for g in range(count)]
+        for gather in (grass.GATHER_AUTO, grass.GATHER_PREPASS, grass.GATHER_IN_CTA, grass.GATHER_COOPERATIVE):
+            opts = dict(gather=gather, token_slices=int(rng.integers(0, 4)))
+            ws = ws_bytes(grass.grass_project_plan(count, T, m, n, r, opts)["workspace_bytes"])
+            ws.fill_(0x3C)
+            Gc = [torch.full((r, n), float("nan"), dtype=torch.float32, device=DEV) for _ in range(count)]
+            grass.grass_project_grad_ex(dYd, Xd, idx, rhod, r, Gc, ws, opts)
+            grass.grass_device_status()
+            for g in range(count):
+                _assert_close_gc(f64(Gc[g]), want[g])
+
+
 def test_cooperative_gather_is_bit_reproducible_and_matches_the_prepass():
     """Same tiling, same token slices: the cooperative gather and the pre-pass feed the GEMM the
     same operand bits, so the results are identical, run after run."""
