@@ -127,7 +127,9 @@ def test_layer_step_on_sampled_rows(case):
     (32768, 11008, 4096, 1024, 2),     # 7B gate, up
     (65536, 2048, 2048, 512, 4),       # 1B q,k,v,o
     (65536, 1024, 1024, 256, 4),       # 350M q,k,v,o
-], ids=["7b_qkvo_r1024", "7b_qkvo_r256", "7b_gateup_r1024", "1b_qkvo_r512", "350m_qkvo_r256"])
+    (32768, 5120, 5120, 1024, 4),      # 13B q,k,v,o: three waves of tiles, long + short token slices
+], ids=["7b_qkvo_r1024", "7b_qkvo_r256", "7b_gateup_r1024", "1b_qkvo_r512", "350m_qkvo_r256",
+        "13b_qkvo_r1024"])
 def test_batched_projection_on_sampled_rows(T, m, n, r, count):
     """Same-shaped projections of a block stepped as one group, as bench.py does: one set of
     launches over `count` layers (a different tiling plan from the single-layer call)."""
